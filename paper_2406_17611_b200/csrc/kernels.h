@@ -1,0 +1,45 @@
+// Launchers of the kernels behind the C ABI (internal).
+#ifndef VARCO_KERNELS_H_
+#define VARCO_KERNELS_H_
+
+#include <cuda_runtime.h>
+
+#include "varco_internal.h"
+
+// workspace carving shared by varco_workspace_bytes and the layer entry points
+struct varco_ws_layout {
+  int64_t ld_in = 0, ld_out = 0;  // leading dimensions of the internal buffers
+  size_t packed = 0, halo = 0, dZ = 0, dAgg = 0, scratch = 0, scratch_bytes = 0, total = 0;
+};
+varco_ws_layout varco_make_ws_layout(const varco_plan *pl, int F_in, int F_out, varco_dtype_t dt);
+size_t varco_gemm_scratch_bytes(int F_in, int F_out);
+
+// halo.cu
+int varco_launch_compress_rows(const varco_plan *pl, const void *X, int64_t ld, int F, int k, varco_dtype_t dt,
+                               varco_key_t key, void *packed, cudaStream_t st);
+int varco_launch_decompress_slots(const varco_plan *pl, const void *packed, int F, int k, varco_dtype_t dt,
+                                  varco_key_t key, void *Xhalo, int64_t ld, cudaStream_t st);
+int varco_launch_compress_slots(const varco_plan *pl, const void *G, int64_t ld, int F, int k, varco_dtype_t dt,
+                                varco_key_t key, void *packed, cudaStream_t st);
+int varco_launch_scatter_add_rows(const varco_plan *pl, const void *packed, int F, int k, varco_dtype_t dt,
+                                  varco_key_t key, void *dX, int64_t ld, cudaStream_t st);
+// spmm.cu
+int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, const void *Xhalo, int64_t ldh, int F,
+                          varco_dtype_t dt, void *Agg, int64_t ldagg, cudaStream_t st);
+int varco_launch_spmm_bwd(const varco_plan *pl, const void *dAgg, int64_t ldd, int F, varco_dtype_t dt, void *dX,
+                          int64_t ldx, int accumulate, void *Ghalo, int64_t ldh, cudaStream_t st);
+// gemm_simt.cu
+size_t varco_simt_dw_scratch_bytes(int F_in, int F_out);
+int varco_simt_gemm_fwd(int n, int F_in, int F_out, varco_dtype_t dt, const void *X, int64_t ldx, const void *Agg,
+                        int64_t lda, const void *Ws, const void *Wn, const float *bias, int relu, void *Y,
+                        int64_t ldy, cudaStream_t st);
+int varco_simt_gemm_dx(int n, int F_in, int F_out, varco_dtype_t dt, const void *dZ, int64_t lddz, const void *W,
+                       void *out, int64_t ldo, cudaStream_t st);
+int varco_simt_gemm_dw(int n, int F_in, int F_out, varco_dtype_t dt, const void *A, int64_t lda, const void *dZ,
+                       int64_t lddz, float *dW, float *scratch, cudaStream_t st);
+int varco_colsum(int n, int F_out, varco_dtype_t dt, const void *dZ, int64_t lddz, float *out, float *scratch,
+                 cudaStream_t st);
+int varco_relu_mask(int n, int F_out, varco_dtype_t dt, const void *Y, int64_t ldy, const void *dY, int64_t lddy,
+                    void *dZ, int64_t lddz, cudaStream_t st);
+
+#endif  // VARCO_KERNELS_H_

@@ -1,0 +1,189 @@
+// Entry points of the layer path: compress / decompress over the plan, layer forward and backward.
+//
+// Forward, per Algorithm 1 of the paper: gather + compress the boundary rows (step 2), put them in
+// the receivers' halo slots decompressed (step 3), aggregate exact local rows and lossy remote
+// rows, transform (Eq. (2)).  Backward mirrors it: transform gradients, transposed aggregation
+// to local rows and halo slots, compress the slot gradients with the forward's key, return them
+// to the owners and add (step 4, "back-propagating errors across machines and through the
+// differentiable compression routine").
+#include <new>
+
+#include "device_common.cuh"
+#include "kernels.h"
+
+namespace {
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_matrix(const void *p, int64_t ld, int F, int V) {
+  if (!p || !aligned16(p) || ld < F || (ld % V) != 0) return VARCO_INVALID_ARG;
+  return VARCO_OK;
+}
+
+int check_desc(const varco_plan *pl, const varco_layer_desc_t *d) {
+  if (!pl || !d) return VARCO_INVALID_ARG;
+  if (d->dtype != VARCO_F32 && d->dtype != VARCO_BF16) return VARCO_INVALID_ARG;
+  if ((int)d->conv != pl->conv) return VARCO_INVALID_ARG;
+  if (d->F_in < 1 || d->F_out < 1) return VARCO_INVALID_ARG;
+  if (d->F_in > 2048 || d->F_out > 2048) return VARCO_UNSUPPORTED;
+  if (!pl->uploaded) return VARCO_NOT_UPLOADED;
+  return VARCO_OK;
+}
+
+}  // namespace
+
+size_t varco_gemm_scratch_bytes(int F_in, int F_out) { return varco_simt_dw_scratch_bytes(F_in, F_out); }
+
+extern "C" {
+
+int varco_compress(const varco_plan_t *plan, const void *X, int64_t ld, int32_t F, varco_dtype_t dtype,
+                   varco_ratio_t c, varco_key_t key, void *packed, uint64_t *bytes, void *stream) {
+  if (!plan || (dtype != VARCO_F32 && dtype != VARCO_BF16)) return VARCO_INVALID_ARG;
+  const int V = dtype == VARCO_F32 ? 4 : 8;
+  const int k = varco_kept_internal(F, c);
+  if (k < 0) return VARCO_INVALID_ARG;
+  if (F > 2048) return VARCO_UNSUPPORTED;
+  if (check_matrix(X, ld, F, V) != VARCO_OK) return VARCO_INVALID_ARG;
+  if (plan->H > 0 && !packed) return VARCO_INVALID_ARG;
+  if (!plan->uploaded) return VARCO_NOT_UPLOADED;
+  if (bytes) *bytes = (uint64_t)plan->H * (uint64_t)k * (dtype == VARCO_F32 ? 4u : 2u);
+  StageTimer t(plan, VARCO_STAGE_COMPRESS, stream);
+  return varco_launch_compress_rows(plan, X, ld, F, k, dtype, key, packed, (cudaStream_t)stream);
+}
+
+int varco_decompress(const varco_plan_t *plan, const void *packed, int32_t F, varco_dtype_t dtype, varco_ratio_t c,
+                     varco_key_t key, void *Xhalo, int64_t ld, void *stream) {
+  if (!plan || (dtype != VARCO_F32 && dtype != VARCO_BF16)) return VARCO_INVALID_ARG;
+  const int V = dtype == VARCO_F32 ? 4 : 8;
+  const int k = varco_kept_internal(F, c);
+  if (k < 0) return VARCO_INVALID_ARG;
+  if (F > 2048) return VARCO_UNSUPPORTED;
+  if (plan->H > 0 && (!packed || check_matrix(Xhalo, ld, F, V) != VARCO_OK)) return VARCO_INVALID_ARG;
+  if (!plan->uploaded) return VARCO_NOT_UPLOADED;
+  StageTimer t(plan, VARCO_STAGE_DECOMPRESS, stream);
+  return varco_launch_decompress_slots(plan, packed, F, k, dtype, key, Xhalo, ld, (cudaStream_t)stream);
+}
+
+int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, const void *X, const void *W_self,
+                    const void *W_neigh, const float *bias, void *Y, void *Agg_saved, varco_ratio_t c,
+                    varco_key_t key, void *workspace, size_t ws_bytes, uint64_t *halo_bytes, void *stream) {
+  int rc = check_desc(plan, desc);
+  if (rc != VARCO_OK) return rc;
+  const varco_dtype_t dt = desc->dtype;
+  const int V = dt == VARCO_F32 ? 4 : 8;
+  const size_t es = dt == VARCO_F32 ? 4 : 2;
+  const int F_in = desc->F_in, F_out = desc->F_out;
+  const int k = varco_kept_internal(F_in, c);
+  if (k < 0) return VARCO_INVALID_ARG;
+  if (check_matrix(X, desc->ld_in, F_in, V) || check_matrix(Agg_saved, desc->ld_in, F_in, V) ||
+      check_matrix(Y, desc->ld_out, F_out, V))
+    return VARCO_INVALID_ARG;
+  if (!W_neigh || (desc->conv == VARCO_SAGE_MEAN && !W_self) || (desc->conv == VARCO_GCN && W_self))
+    return VARCO_INVALID_ARG;
+  if (!workspace || !aligned16(workspace)) return VARCO_INVALID_ARG;
+  const varco_ws_layout L = varco_make_ws_layout(plan, F_in, F_out, dt);
+  if (ws_bytes < L.total) return VARCO_WORKSPACE_TOO_SMALL;
+  char *ws = static_cast<char *>(workspace);
+  ws += (256 - (reinterpret_cast<uintptr_t>(ws) & 255u)) & 255u;
+  void *packed = ws + L.packed;
+  void *Xhalo = ws + L.halo;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (halo_bytes) *halo_bytes = (uint64_t)plan->H * (uint64_t)k * es;
+
+  {
+    StageTimer t(plan, VARCO_STAGE_COMPRESS, stream);
+    rc = varco_launch_compress_rows(plan, X, desc->ld_in, F_in, k, dt, key, packed, st);
+  }
+  if (rc != VARCO_OK) return rc;
+  {
+    StageTimer t(plan, VARCO_STAGE_DECOMPRESS, stream);
+    rc = varco_launch_decompress_slots(plan, packed, F_in, k, dt, key, Xhalo, L.ld_in, st);
+  }
+  if (rc != VARCO_OK) return rc;
+  {
+    StageTimer t(plan, VARCO_STAGE_SPMM, stream);
+    rc = varco_launch_spmm_fwd(plan, X, desc->ld_in, Xhalo, L.ld_in, F_in, dt, Agg_saved, desc->ld_in, st);
+  }
+  if (rc != VARCO_OK) return rc;
+  {
+    StageTimer t(plan, VARCO_STAGE_GEMM_FWD, stream);
+    rc = varco_simt_gemm_fwd((int)plan->n, F_in, F_out, dt, X, desc->ld_in, Agg_saved, desc->ld_in, W_self, W_neigh,
+                             bias, desc->relu, Y, desc->ld_out, st);
+  }
+  return rc;
+}
+
+int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, const void *X, const void *Y,
+                    const void *Agg_saved, const void *W_self, const void *W_neigh, const void *dY, void *dX,
+                    float *dW_self, float *dW_neigh, float *dbias, varco_ratio_t c, varco_key_t key, void *workspace,
+                    size_t ws_bytes, uint64_t *halo_bytes, void *stream) {
+  int rc = check_desc(plan, desc);
+  if (rc != VARCO_OK) return rc;
+  const varco_dtype_t dt = desc->dtype;
+  const int V = dt == VARCO_F32 ? 4 : 8;
+  const size_t es = dt == VARCO_F32 ? 4 : 2;
+  const int F_in = desc->F_in, F_out = desc->F_out;
+  const int n = (int)plan->n;
+  const bool sage = desc->conv == VARCO_SAGE_MEAN;
+  const int k = varco_kept_internal(F_in, c);
+  if (k < 0) return VARCO_INVALID_ARG;
+  if (check_matrix(X, desc->ld_in, F_in, V) || check_matrix(Agg_saved, desc->ld_in, F_in, V) ||
+      check_matrix(dX, desc->ld_in, F_in, V) || check_matrix(dY, desc->ld_out, F_out, V))
+    return VARCO_INVALID_ARG;
+  if (desc->relu && check_matrix(Y, desc->ld_out, F_out, V)) return VARCO_INVALID_ARG;
+  if (!W_neigh || !dW_neigh || (sage && (!W_self || !dW_self)) || (!sage && (W_self || dW_self)))
+    return VARCO_INVALID_ARG;
+  if (!workspace || !aligned16(workspace)) return VARCO_INVALID_ARG;
+  const varco_ws_layout L = varco_make_ws_layout(plan, F_in, F_out, dt);
+  if (ws_bytes < L.total) return VARCO_WORKSPACE_TOO_SMALL;
+  char *ws = static_cast<char *>(workspace);
+  ws += (256 - (reinterpret_cast<uintptr_t>(ws) & 255u)) & 255u;
+  void *packed = ws + L.packed;
+  void *Ghalo = ws + L.halo;
+  void *dZbuf = ws + L.dZ;
+  void *dAgg = ws + L.dAgg;
+  float *scratch = reinterpret_cast<float *>(ws + L.scratch);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (halo_bytes) *halo_bytes = (uint64_t)plan->H * (uint64_t)k * es;
+
+  const void *dZ = dY;
+  int64_t lddz = desc->ld_out;
+  if (desc->relu) {
+    StageTimer t(plan, VARCO_STAGE_AUX, stream);
+    rc = varco_relu_mask(n, F_out, dt, Y, desc->ld_out, dY, desc->ld_out, dZbuf, L.ld_out, st);
+    if (rc != VARCO_OK) return rc;
+    dZ = dZbuf;
+    lddz = L.ld_out;
+  }
+  {
+    StageTimer t(plan, VARCO_STAGE_GEMM_DW, stream);
+    rc = varco_simt_gemm_dw(n, F_in, F_out, dt, Agg_saved, desc->ld_in, dZ, lddz, dW_neigh, scratch, st);
+    if (rc == VARCO_OK && sage)
+      rc = varco_simt_gemm_dw(n, F_in, F_out, dt, X, desc->ld_in, dZ, lddz, dW_self, scratch, st);
+    if (rc == VARCO_OK && dbias) rc = varco_colsum(n, F_out, dt, dZ, lddz, dbias, scratch, st);
+  }
+  if (rc != VARCO_OK) return rc;
+  {
+    StageTimer t(plan, VARCO_STAGE_GEMM_DX, stream);
+    rc = varco_simt_gemm_dx(n, F_in, F_out, dt, dZ, lddz, W_neigh, dAgg, L.ld_in, st);
+    if (rc == VARCO_OK && sage) rc = varco_simt_gemm_dx(n, F_in, F_out, dt, dZ, lddz, W_self, dX, desc->ld_in, st);
+  }
+  if (rc != VARCO_OK) return rc;
+  {
+    StageTimer t(plan, VARCO_STAGE_SPMM_T, stream);
+    rc = varco_launch_spmm_bwd(plan, dAgg, L.ld_in, F_in, dt, dX, desc->ld_in, sage ? 1 : 0, Ghalo, L.ld_in, st);
+  }
+  if (rc != VARCO_OK) return rc;
+  {
+    StageTimer t(plan, VARCO_STAGE_COMPRESS_BWD, stream);
+    rc = varco_launch_compress_slots(plan, Ghalo, L.ld_in, F_in, k, dt, key, packed, st);
+  }
+  if (rc != VARCO_OK) return rc;
+  {
+    StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
+    rc = varco_launch_scatter_add_rows(plan, packed, F_in, k, dt, key, dX, desc->ld_in, st);
+  }
+  return rc;
+}
+
+}  // extern "C"

@@ -1,0 +1,207 @@
+// Device image of the plan, workspace sizing and per-stage event timing.
+#include <mutex>
+
+#include "device_common.cuh"
+#include "kernels.h"
+
+namespace {
+
+struct ImageItem {
+  const void *host;
+  size_t bytes;
+  const void **dev;
+};
+
+template <typename T> ImageItem item(const std::vector<T> &v, const T **dev) {
+  return ImageItem{v.data(), v.size() * sizeof(T), reinterpret_cast<const void **>(dev)};
+}
+
+std::vector<ImageItem> image_items(varco_plan *pl) {
+  varco_dev_image &d = pl->d;
+  return {item(pl->row_gid, &d.row_gid),
+          item(pl->rp, &d.rp),
+          item(pl->col, &d.col),
+          item(pl->val, &d.val),
+          item(pl->rpT, &d.rpT),
+          item(pl->colT, &d.colT),
+          item(pl->valT, &d.valT),
+          item(pl->slot_gid, &d.slot_gid),
+          item(pl->slot_src, &d.slot_src),
+          item(pl->slot_sendpos, &d.slot_sendpos),
+          item(pl->brow, &d.brow),
+          item(pl->brow_ptr, &d.brow_ptr),
+          item(pl->brow_slot, &d.brow_slot),
+          item(pl->order_f, &d.order_f),
+          item(pl->order_t, &d.order_t)};
+}
+
+size_t aligned(size_t b) { return (b + 255) / 256 * 256; }
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------ profile
+struct varco_profile {
+  bool on = false;
+  std::mutex mu;
+  struct Span {
+    cudaEvent_t a, b;
+  };
+  std::vector<Span> spans[VARCO_STAGE_COUNT];
+  std::vector<Span> pool;
+  Span open[VARCO_STAGE_COUNT];
+  bool is_open[VARCO_STAGE_COUNT] = {};
+};
+
+void varco_prof_begin(const varco_plan *plan, int stage, void *stream) {
+  varco_profile *pr = plan->prof;
+  if (!pr || !pr->on) return;
+  std::lock_guard<std::mutex> lock(pr->mu);
+  varco_profile::Span s;
+  if (!pr->pool.empty()) {
+    s = pr->pool.back();
+    pr->pool.pop_back();
+  } else {
+    if (cudaEventCreate(&s.a) != cudaSuccess) return;
+    if (cudaEventCreate(&s.b) != cudaSuccess) {
+      cudaEventDestroy(s.a);
+      return;
+    }
+  }
+  cudaEventRecord(s.a, (cudaStream_t)stream);
+  pr->open[stage] = s;
+  pr->is_open[stage] = true;
+}
+
+void varco_prof_end(const varco_plan *plan, int stage, void *stream) {
+  varco_profile *pr = plan->prof;
+  if (!pr || !pr->on) return;
+  std::lock_guard<std::mutex> lock(pr->mu);
+  if (!pr->is_open[stage]) return;
+  cudaEventRecord(pr->open[stage].b, (cudaStream_t)stream);
+  pr->spans[stage].push_back(pr->open[stage]);
+  pr->is_open[stage] = false;
+}
+
+void varco_prof_destroy(varco_plan *plan) {
+  varco_profile *pr = plan->prof;
+  if (!pr) return;
+  for (int s = 0; s < VARCO_STAGE_COUNT; ++s)
+    for (auto &sp : pr->spans[s]) {
+      cudaEventDestroy(sp.a);
+      cudaEventDestroy(sp.b);
+    }
+  for (auto &sp : pr->pool) {
+    cudaEventDestroy(sp.a);
+    cudaEventDestroy(sp.b);
+  }
+  delete pr;
+  plan->prof = nullptr;
+}
+
+extern "C" {
+
+int varco_profile_enable(varco_plan_t *plan, int on) {
+  if (!plan) return VARCO_INVALID_ARG;
+  if (!plan->prof) plan->prof = new (std::nothrow) varco_profile;
+  if (!plan->prof) return VARCO_NOMEM;
+  plan->prof->on = on != 0;
+  return VARCO_OK;
+}
+
+int varco_profile_reset(varco_plan_t *plan) {
+  if (!plan) return VARCO_INVALID_ARG;
+  varco_profile *pr = plan->prof;
+  if (!pr) return VARCO_OK;
+  std::lock_guard<std::mutex> lock(pr->mu);
+  for (int s = 0; s < VARCO_STAGE_COUNT; ++s) {
+    for (auto &sp : pr->spans[s]) {
+      cudaEventSynchronize(sp.b);
+      pr->pool.push_back(sp);
+    }
+    pr->spans[s].clear();
+  }
+  return VARCO_OK;
+}
+
+int varco_profile_read(varco_plan_t *plan, int64_t *launches, double *milliseconds) {
+  if (!plan || !launches || !milliseconds) return VARCO_INVALID_ARG;
+  for (int s = 0; s < VARCO_STAGE_COUNT; ++s) {
+    launches[s] = 0;
+    milliseconds[s] = 0.0;
+  }
+  varco_profile *pr = plan->prof;
+  if (!pr) return VARCO_OK;
+  std::lock_guard<std::mutex> lock(pr->mu);
+  for (int s = 0; s < VARCO_STAGE_COUNT; ++s)
+    for (auto &sp : pr->spans[s]) {
+      VARCO_CUDA_CHECK(cudaEventSynchronize(sp.b));
+      float ms = 0.f;
+      VARCO_CUDA_CHECK(cudaEventElapsedTime(&ms, sp.a, sp.b));
+      launches[s] += 1;
+      milliseconds[s] += (double)ms;
+    }
+  return VARCO_OK;
+}
+
+// ------------------------------------------------------------------------------------------ image
+int varco_partition_device_bytes(const varco_plan_t *plan, size_t *bytes) {
+  if (!plan || !bytes) return VARCO_INVALID_ARG;
+  size_t total = 0;
+  for (const ImageItem &it : image_items(const_cast<varco_plan *>(plan))) total += aligned(it.bytes);
+  *bytes = total + 256;
+  return VARCO_OK;
+}
+
+int varco_partition_upload(varco_plan_t *plan, void *dev_buf, size_t bytes, void *stream) {
+  if (!plan || !dev_buf) return VARCO_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(dev_buf) & 255u) != 0) return VARCO_INVALID_ARG;
+  size_t need = 0;
+  varco_partition_device_bytes(plan, &need);
+  if (bytes < need) return VARCO_WORKSPACE_TOO_SMALL;
+  plan->uploaded = false;
+  size_t off = 0;
+  for (const ImageItem &it : image_items(plan)) {
+    char *dst = static_cast<char *>(dev_buf) + off;
+    if (it.bytes)
+      VARCO_CUDA_CHECK(cudaMemcpyAsync(dst, it.host, it.bytes, cudaMemcpyHostToDevice, (cudaStream_t)stream));
+    *it.dev = dst;
+    off += aligned(it.bytes);
+  }
+  VARCO_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream));
+  plan->uploaded = true;
+  return VARCO_OK;
+}
+
+int varco_workspace_bytes(const varco_plan_t *plan, int32_t F_in_max, int32_t F_out_max, varco_dtype_t dtype,
+                          size_t *bytes) {
+  if (!plan || !bytes || F_in_max < 1 || F_out_max < 1 || (dtype != VARCO_F32 && dtype != VARCO_BF16))
+    return VARCO_INVALID_ARG;
+  if (F_in_max > 2048 || F_out_max > 2048) return VARCO_UNSUPPORTED;
+  varco_ws_layout L = varco_make_ws_layout(plan, F_in_max, F_out_max, dtype);
+  *bytes = L.total;
+  return VARCO_OK;
+}
+
+}  // extern "C"
+
+varco_ws_layout varco_make_ws_layout(const varco_plan *pl, int F_in, int F_out, varco_dtype_t dt) {
+  const size_t es = dt == VARCO_F32 ? 4 : 2;
+  const int V = 16 / (int)es;
+  varco_ws_layout L;
+  L.ld_in = round_up64(F_in, V);
+  L.ld_out = round_up64(F_out, V);
+  size_t off = 0;
+  auto take = [&](size_t b) {
+    size_t o = off;
+    off += aligned(b);
+    return o;
+  };
+  L.packed = take((size_t)pl->H * F_in * es);
+  L.halo = take((size_t)pl->H * L.ld_in * es);      // forward: decompressed rows; backward: slot gradients
+  L.dZ = take((size_t)pl->n * L.ld_out * es);
+  L.dAgg = take((size_t)pl->n * L.ld_in * es);
+  L.scratch_bytes = varco_gemm_scratch_bytes(F_in, F_out);
+  L.scratch = take(L.scratch_bytes);
+  L.total = off + 256;
+  return L;
+}

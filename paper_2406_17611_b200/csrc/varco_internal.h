@@ -1,0 +1,70 @@
+// Internal declarations of libvarco: the plan object and the kernel launchers.
+#ifndef VARCO_INTERNAL_H_
+#define VARCO_INTERNAL_H_
+
+#include <cstddef>
+#include <cstdint>
+#include <vector>
+
+#include "varco.h"
+
+struct varco_dev_image {
+  // row r of the partition-contiguous order -> original node id (the id the keys are derived from)
+  const int32_t *row_gid = nullptr;
+  // aggregation structure of all partitions: row r aggregates from sources col[e] with weight
+  // val[e]; a source < n is the local row of X with that index, a source >= n is halo slot (col - n)
+  const int64_t *rp = nullptr;
+  const int32_t *col = nullptr;
+  const float *val = nullptr;
+  // transposed structure: source u (row or n + slot) is used by rows colT[e] with weight valT[e]
+  const int64_t *rpT = nullptr;
+  const int32_t *colT = nullptr;
+  const float *valT = nullptr;
+  // halo slots in receive order (destination, owner, id)
+  const int32_t *slot_gid = nullptr;      // original id of the source node
+  const int32_t *slot_src = nullptr;      // row of X that owns the data
+  const int32_t *slot_sendpos = nullptr;  // position of the copy in send order (owner, destination, id)
+  // unique boundary rows and the slots each one feeds (ascending destination)
+  const int32_t *brow = nullptr;
+  const int32_t *brow_ptr = nullptr;
+  const int32_t *brow_slot = nullptr;
+  // rows sorted by descending number of entries (forward rows; transposed sources)
+  const int32_t *order_f = nullptr;
+  const int32_t *order_t = nullptr;
+};
+
+struct varco_profile;  // CUDA-event bookkeeping, defined in runtime.cu
+
+struct varco_plan {
+  int64_t n = 0, nnz = 0, nnz_f = 0, H = 0, cross = 0, self_ = 0, nb = 0;
+  int32_t P = 0;
+  int conv = 0;
+  std::vector<int64_t> new_to_old, part_off, counts, send_base, halo_ids;
+  // host copies of the device image
+  std::vector<int32_t> row_gid, col, colT, slot_gid, slot_src, slot_sendpos, brow, brow_ptr, brow_slot;
+  std::vector<int32_t> order_f, order_t;
+  std::vector<int64_t> rp, rpT;
+  std::vector<float> val, valT;
+  // device image
+  bool uploaded = false;
+  varco_dev_image d;
+  varco_profile *prof = nullptr;
+};
+
+// rate helpers shared by the entry points
+int varco_kept_internal(int32_t F, varco_ratio_t c);
+
+// profile hooks (runtime.cu)
+void varco_prof_begin(const varco_plan *plan, int stage, void *stream);
+void varco_prof_end(const varco_plan *plan, int stage, void *stream);
+void varco_prof_destroy(varco_plan *plan);
+
+struct StageTimer {
+  const varco_plan *plan;
+  int stage;
+  void *stream;
+  StageTimer(const varco_plan *p, int s, void *st) : plan(p), stage(s), stream(st) { varco_prof_begin(p, s, st); }
+  ~StageTimer() { varco_prof_end(plan, stage, stream); }
+};
+
+#endif  // VARCO_INTERNAL_H_

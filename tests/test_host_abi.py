@@ -1,0 +1,100 @@
+"""Host-side checks of the C-ABI library: exported symbols, plan builder against the oracle's
+partition sets (bit-exact), rate helpers, error codes.  No GPU needed."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2406_17611_b200 import binding as vb
+from paper_2406_17611_b200 import build as vbuild
+from paper_2406_17611_b200 import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    vbuild.build()
+
+
+def test_library_exports_every_declared_symbol():
+    text = open(os.path.join(ROOT, "include", "varco.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = sorted(set(re.findall(r"\b(varco_[a-z_0-9]+)\s*\(", text)))
+    assert len(declared) >= 19
+    L = C.CDLL(vb.LIB_PATH)
+    for name in declared:
+        assert hasattr(L, name), name
+    assert sorted(vb.EXPORTS) == declared
+
+
+@pytest.mark.parametrize("name,scale", [("c1", 1.0), ("c2", 0.05), ("c2r", 0.05), ("c3", 0.004), ("c4", 0.02)])
+def test_plan_matches_oracle_partition_bit_exact(orc, name, scale):
+    wl = synth.make_workload(name, scale)
+    plan = vb.Plan(wl.row_ptr, wl.col, wl.part, wl.parts, wl.conv)
+    g = orc.graph(wl.row_ptr, wl.col, wl.part, wl.parts, wl.conv)
+    assert (plan.n, plan.nnz, plan.P) == (wl.n, wl.nnz, wl.parts)
+    assert plan.H_total == g.H_total
+    assert plan.cross_entries == g.cross_entries and plan.self_entries == g.self_entries
+    assert np.array_equal(plan.counts(), g.counts())
+    assert np.array_equal(plan.perm(), g.perm())
+    for p in range(wl.parts):
+        for q in range(wl.parts):
+            assert np.array_equal(plan.halo(p, q), g.halo(p, q))
+    plan.close()
+
+
+def test_rate_helpers_match_oracle(orc):
+    for F in (1, 47, 64, 100, 256, 602):
+        for K, a in [(20, 5), (100, 5), (300, 5), (300, 2), (300, 7)]:
+            for e in range(0, K, max(1, K // 23)):
+                r = vb.varco_schedule_linear(e, K, a)
+                assert r == orc.schedule_linear(e, K, a)
+                assert vb.varco_kept(F, r) == orc.kept(F, r)
+    # worked values: K=100, a=5 -> c_e = 128 - 6.35 e; F=256 keeps 2, 3, ... 35 (e=19), 256 (e>=20)
+    ks = [vb.varco_kept(256, vb.varco_schedule_linear(e, 100)) for e in range(22)]
+    assert ks[0] == 2 and ks[1] == 3 and ks[19] == 35 and ks[20] == ks[21] == 256
+    assert vb.varco_kept(256, vb.varco_schedule_linear(59, 300)) == 83
+
+
+def test_error_codes():
+    L = vb.lib()
+    rp = np.array([0, 1, 2], dtype=np.int64)
+    col = np.array([1, 0], dtype=np.int32)
+    part = np.array([0, 1], dtype=np.int32)
+
+    def build(rp, col, part, P=2, conv=1):
+        h = C.c_void_p()
+        st = L.varco_partition_build(len(rp) - 1, rp.ctypes.data_as(C.POINTER(C.c_int64)),
+                                     col.ctypes.data_as(C.POINTER(C.c_int32)),
+                                     part.ctypes.data_as(C.POINTER(C.c_int32)), P, conv, C.byref(h))
+        if st == 0:
+            L.varco_partition_destroy(h)
+        return st
+    assert build(rp, col, part) == 0
+    assert build(np.array([0, 2, 1], dtype=np.int64), col, part) == -2          # row_ptr not monotone
+    assert build(np.array([1, 1, 2], dtype=np.int64), col, part) == -2          # does not start at 0
+    assert build(rp, np.array([2, 0], dtype=np.int32), part) == -2              # column out of range
+    assert build(rp, np.array([0, 0], dtype=np.int32), part) == -2              # diagonal entry
+    assert build(np.array([0, 2, 2], dtype=np.int64), np.array([1, 1], dtype=np.int32), part) == -2   # duplicate
+    assert build(rp, col, np.array([0, 2], dtype=np.int32)) == -3               # label out of range
+    assert build(rp, col, part, P=0) == -1
+    assert build(rp, col, part, conv=5) == -1
+    with pytest.raises(vb.VarcoError):
+        vb.varco_kept(64, (1, 2))
+    with pytest.raises(vb.VarcoError):
+        vb.varco_schedule_linear(0, 0)
+    assert L.varco_status_string(-6) == b"workspace too small"
+    # device entry points refuse a plan that has no device image, without touching the GPU
+    plan = vb.Plan(rp, col, part, 2, "sage")
+    d = vb.LayerDesc(1, 0, 4, 4, 1, 4, 4)
+    buf = (C.c_float * 64)()
+    st = L.varco_layer_fwd(plan.h, C.byref(d), buf, buf, buf, None, buf, buf, vb.Ratio(1, 1), vb.Key(0, 0, 0), buf,
+                           1 << 20, None, None)
+    assert st == -8
+    nbytes = C.c_size_t()
+    assert L.varco_workspace_bytes(plan.h, 4096, 4, 0, C.byref(nbytes)) == -7
+    assert L.varco_workspace_bytes(plan.h, 64, 64, 0, C.byref(nbytes)) == 0 and nbytes.value > 0
+    plan.close()
