@@ -96,6 +96,8 @@ int varco_partition_destroy(varco_plan_t *plan);
  *   cross_entries  stored entries (i, j) with part(i) != part(j); self_entries the others. */
 int varco_partition_info(const varco_plan_t *plan, int64_t *n, int64_t *nnz, int32_t *P,
                          int64_t *H_total, int64_t *cross_entries, int64_t *self_entries);
+/* Number of distinct rows that are a halo row of at least one other partition. */
+int varco_partition_boundary_rows(const varco_plan_t *plan, int64_t *count);
 /* PxP[p * P + q] = |halo(p->q)| (host array of P*P entries). */
 int varco_partition_counts(const varco_plan_t *plan, int64_t *PxP);
 /* Original ids of halo(p->q), ascending; the pointer stays valid until the plan is destroyed. */
@@ -207,7 +209,7 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
  * Per-stage device timing (no counterpart in the paper; a measurement aid).
  * When enabled, every kernel stage of the entry points above is bracketed by CUDA events on the
  * stream it is launched on.  varco_profile_read synchronises those events and returns, per stage,
- * the number of launches and the summed milliseconds since the last reset.
+ * the number of timed stage executions and the summed milliseconds since the last reset.
  */
 enum {
   VARCO_STAGE_COMPRESS = 0,      /* halo gather + compress (forward)            */
@@ -226,6 +228,9 @@ int varco_profile_enable(varco_plan_t *plan, int on);
 int varco_profile_reset(varco_plan_t *plan);
 int varco_profile_read(varco_plan_t *plan, int64_t *launches /* [VARCO_STAGE_COUNT] */,
                        double *milliseconds /* [VARCO_STAGE_COUNT] */);
+/* Number of CUDA kernels this library has launched in this process so far (all plans, all
+ * streams).  Also a measurement aid without a counterpart in the paper. */
+int varco_kernel_launches(int64_t *count);
 
 #ifdef __cplusplus
 }

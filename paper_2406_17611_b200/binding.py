@@ -20,10 +20,10 @@ STAGES = ["compress", "decompress", "spmm", "gemm_fwd", "gemm_dx", "gemm_dw", "s
           "scatter_add", "aux"]
 
 EXPORTS = ["varco_status_string", "varco_partition_build", "varco_partition_destroy", "varco_partition_info",
-           "varco_partition_counts", "varco_partition_halo", "varco_partition_perm", "varco_partition_device_bytes",
+           "varco_partition_boundary_rows", "varco_partition_counts", "varco_partition_halo", "varco_partition_perm", "varco_partition_device_bytes",
            "varco_partition_upload", "varco_workspace_bytes", "varco_kept", "varco_schedule_linear",
            "varco_compress", "varco_decompress", "varco_layer_fwd", "varco_layer_bwd", "varco_profile_enable",
-           "varco_profile_reset", "varco_profile_read"]
+           "varco_profile_reset", "varco_profile_read", "varco_kernel_launches"]
 
 
 class Ratio(C.Structure):
@@ -64,6 +64,7 @@ def lib():
     L.varco_partition_destroy.argtypes = [vp]
     L.varco_partition_info.argtypes = [vp, i64p, i64p, i32p, i64p, i64p, i64p]
     L.varco_partition_counts.argtypes = [vp, i64p]
+    L.varco_partition_boundary_rows.argtypes = [vp, i64p]
     L.varco_partition_halo.argtypes = [vp, C.c_int32, C.c_int32, C.POINTER(i64p), i64p]
     L.varco_partition_perm.argtypes = [vp, C.POINTER(i64p)]
     L.varco_partition_device_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
@@ -80,6 +81,7 @@ def lib():
     L.varco_profile_enable.argtypes = [vp, C.c_int]
     L.varco_profile_reset.argtypes = [vp]
     L.varco_profile_read.argtypes = [vp, i64p, C.POINTER(C.c_double)]
+    L.varco_kernel_launches.argtypes = [i64p]
     _lib = L
     return L
 
@@ -120,6 +122,12 @@ def varco_schedule_linear(epoch, K, slope_a=5, c_max=128, c_min=1):
     return (int(r.num), int(r.den))
 
 
+def varco_kernel_launches():
+    c = C.c_int64()
+    _check(lib().varco_kernel_launches(C.byref(c)), "varco_kernel_launches")
+    return int(c.value)
+
+
 class Plan:
     """varco_partition_build and friends.  Owns the plan handle and (after upload) its device image."""
 
@@ -141,6 +149,9 @@ class Plan:
                                           C.byref(self_e)), "varco_partition_info")
         self.n, self.nnz, self.P, self.H_total = int(n_.value), int(nnz.value), int(P_.value), int(H.value)
         self.cross_entries, self.self_entries = int(cross.value), int(self_e.value)
+        nb = C.c_int64()
+        _check(lib().varco_partition_boundary_rows(self.h, C.byref(nb)), "varco_partition_boundary_rows")
+        self.boundary_rows = int(nb.value)
 
     def close(self):
         if self.h:

@@ -14,6 +14,14 @@
     if (e__ != cudaSuccess) return VARCO_CUDA;   \
   } while (0)
 
+// every kernel launch of the library goes through this: count it, then check the launch status
+void varco_count_launch();
+#define VARCO_KERNEL_LAUNCHED()                  \
+  do {                                           \
+    varco_count_launch();                        \
+    VARCO_CUDA_CHECK(cudaGetLastError());        \
+  } while (0)
+
 // ------------------------------------------------------------------------------------------
 // Shared-key permutation of [0, F): which positions of a row are sent (appendix "Compression
 // Mechanism": chosen at random at the encoder, known to the decoder through a shared key).

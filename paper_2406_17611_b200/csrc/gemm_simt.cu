@@ -157,7 +157,7 @@ int fwd_t(int n, int F_in, int F_out, const T *X, int64_t ldx, const T *Agg, int
   dim3 grid((n + BM - 1) / BM, (F_out + BN - 1) / BN, 1);
   Operand<T> pa{Agg, lda, Wn, F_out, F_in}, px{X, ldx, Ws, F_out, F_in};
   gemm_kernel<T, T, false, false><<<grid, 256, 0, st>>>(n, F_out, pa, px, Ws ? 2 : 1, bias, relu, Y, ldy, 0);
-  VARCO_CUDA_CHECK(cudaGetLastError());
+  VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
@@ -166,7 +166,7 @@ int dx_t(int n, int F_in, int F_out, const T *dZ, int64_t lddz, const T *W, T *o
   dim3 grid((n + BM - 1) / BM, (F_in + BN - 1) / BN, 1);
   Operand<T> p{dZ, lddz, W, F_out, F_out};
   gemm_kernel<T, T, false, true><<<grid, 256, 0, st>>>(n, F_in, p, p, 1, nullptr, 0, out, ldo, 0);
-  VARCO_CUDA_CHECK(cudaGetLastError());
+  VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
@@ -214,10 +214,10 @@ static int dw_t(int n, int F_in, int F_out, const T *A, int64_t lda, const T *dZ
   dim3 grid((F_in + BM - 1) / BM, (F_out + BN - 1) / BN, splits);
   Operand<T> p{A, lda, dZ, lddz, n};
   gemm_kernel<T, float, true, false><<<grid, 256, 0, st>>>(F_in, F_out, p, p, 1, nullptr, 0, scratch, F_out, chunk);
-  VARCO_CUDA_CHECK(cudaGetLastError());
+  VARCO_KERNEL_LAUNCHED();
   const int64_t count = (int64_t)F_in * F_out;
   reduce_partials_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(scratch, count, splits, dW);
-  VARCO_CUDA_CHECK(cudaGetLastError());
+  VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
@@ -239,9 +239,9 @@ int varco_colsum(int n, int F_out, varco_dtype_t dt, const void *dZ, int64_t ldd
     colsum_kernel<float><<<grid, 128, 0, st>>>((const float *)dZ, lddz, n, F_out, chunk, scratch);
   else
     colsum_kernel<__nv_bfloat16><<<grid, 128, 0, st>>>((const __nv_bfloat16 *)dZ, lddz, n, F_out, chunk, scratch);
-  VARCO_CUDA_CHECK(cudaGetLastError());
+  VARCO_KERNEL_LAUNCHED();
   reduce_partials_kernel<<<(F_out + 255) / 256, 256, 0, st>>>(scratch, F_out, splits, out);
-  VARCO_CUDA_CHECK(cudaGetLastError());
+  VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
@@ -257,6 +257,6 @@ int varco_relu_mask(int n, int F_out, varco_dtype_t dt, const void *Y, int64_t l
   else
     relu_mask_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16 *)Y, ldy, (const __nv_bfloat16 *)dY,
                                                           lddy, (__nv_bfloat16 *)dZ, lddz, n, nv);
-  VARCO_CUDA_CHECK(cudaGetLastError());
+  VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }

@@ -182,7 +182,7 @@ int varco_launch_compress_rows(const varco_plan *pl, const void *X, int64_t ld, 
     compress_rows_kernel<uint16_t><<<grid, block, row_bytes * wpb, st>>>(
         (const uint16_t *)X, ld, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot, pl->d.slot_sendpos,
         pl->d.row_gid, (int)pl->nb, (uint16_t *)packed);
-  VARCO_CUDA_CHECK(cudaGetLastError());
+  VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
@@ -204,7 +204,7 @@ int varco_launch_decompress_slots(const varco_plan *pl, const void *packed, int 
     decompress_slots_kernel<uint16_t><<<grid, block, row_bytes * wpb, st>>>(
         (const uint16_t *)packed, F, k, h, lkey, pl->d.slot_gid, pl->d.slot_sendpos, (int)pl->H, (uint16_t *)Xhalo,
         ld);
-  VARCO_CUDA_CHECK(cudaGetLastError());
+  VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
@@ -224,7 +224,7 @@ int varco_launch_compress_slots(const varco_plan *pl, const void *G, int64_t ld,
   else
     compress_slots_kernel<uint16_t><<<grid, block, row_bytes * wpb, st>>>(
         (const uint16_t *)G, ld, F, k, h, lkey, pl->d.slot_gid, (int)pl->H, (uint16_t *)packed);
-  VARCO_CUDA_CHECK(cudaGetLastError());
+  VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
@@ -245,6 +245,6 @@ int varco_launch_scatter_add_rows(const varco_plan *pl, const void *packed, int 
     scatter_add_rows_kernel<__nv_bfloat16><<<grid, block, row_bytes * wpb, st>>>(
         (const __nv_bfloat16 *)packed, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot, pl->d.row_gid,
         (int)pl->nb, (__nv_bfloat16 *)dX, ld);
-  VARCO_CUDA_CHECK(cudaGetLastError());
+  VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }

@@ -305,6 +305,12 @@ int varco_partition_info(const varco_plan_t *plan, int64_t *n, int64_t *nnz, int
   return VARCO_OK;
 }
 
+int varco_partition_boundary_rows(const varco_plan_t *plan, int64_t *count) {
+  if (!plan || !count) return VARCO_INVALID_ARG;
+  *count = plan->nb;
+  return VARCO_OK;
+}
+
 int varco_partition_counts(const varco_plan_t *plan, int64_t *PxP) {
   if (!plan || !PxP) return VARCO_INVALID_ARG;
   std::copy(plan->counts.begin(), plan->counts.end(), PxP);

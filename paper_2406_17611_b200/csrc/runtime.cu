@@ -1,5 +1,7 @@
 // Device image of the plan, workspace sizing and per-stage event timing.
+#include <atomic>
 #include <mutex>
+#include <new>
 
 #include "device_common.cuh"
 #include "kernels.h"
@@ -37,7 +39,11 @@ std::vector<ImageItem> image_items(varco_plan *pl) {
 
 size_t aligned(size_t b) { return (b + 255) / 256 * 256; }
 
+std::atomic<int64_t> g_kernel_launches{0};
+
 }  // namespace
+
+void varco_count_launch() { g_kernel_launches.fetch_add(1, std::memory_order_relaxed); }
 
 // ------------------------------------------------------------------------------------------ profile
 struct varco_profile {
@@ -140,6 +146,12 @@ int varco_profile_read(varco_plan_t *plan, int64_t *launches, double *millisecon
       launches[s] += 1;
       milliseconds[s] += (double)ms;
     }
+  return VARCO_OK;
+}
+
+int varco_kernel_launches(int64_t *count) {
+  if (!count) return VARCO_INVALID_ARG;
+  *count = g_kernel_launches.load(std::memory_order_relaxed);
   return VARCO_OK;
 }
 

@@ -126,7 +126,7 @@ int launch(const SpmmArgs &a, cudaStream_t st) {
   spmm_kernel<T, G, NCH, UNR><<<grid, threads, 0, st>>>(a.rp, a.col, a.val, a.order, a.nrows, (const T *)a.A0, a.lda0,
                                                         (const T *)a.A1, a.lda1, a.src_split, (T *)a.O0, a.ldo0,
                                                         (T *)a.O1, a.ldo1, a.dst_split, a.accumulate0, a.nv);
-  VARCO_CUDA_CHECK(cudaGetLastError());
+  VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 

@@ -86,17 +86,28 @@ def _chung_lu(n: int, w: np.ndarray, m: int, rng):
 def chung_lu_power_law(n: int, undirected_edges: int, exponent: float, seed: int):
     """Chung-Lu graph with expected degrees w_i ~ (i + i0)^(-1/(exponent-1)).
 
-    i0 is chosen so that the largest expected degree stays below sqrt(sum w),
-    the usual condition for the Chung-Lu model to be well defined.
+    Endpoints are drawn from the continuous density proportional to (x + i0)^-alpha on [0, n)
+    by inverting its CDF in closed form, then floored to a node index.  i0 = n / 2450 keeps the
+    largest expected degree near sqrt(sum w), the usual Chung-Lu condition.
     """
     rng = np.random.default_rng(seed)
     alpha = 1.0 / (exponent - 1.0)
     i0 = max(1.0, n / 2450.0)
-    w = (np.arange(n, dtype=np.float64) + i0) ** (-alpha)
-    w *= 2.0 * undirected_edges / w.sum()
-    cap = np.sqrt(w.sum())
-    np.minimum(w, cap, out=w)
-    return _chung_lu(n, w, undirected_edges, rng)
+    lo, hi = i0 ** (1.0 - alpha), (n + i0) ** (1.0 - alpha)
+
+    def draw(m):
+        x = rng.random(m)
+        x *= hi - lo
+        x += lo
+        np.power(x, 1.0 / (1.0 - alpha), out=x)
+        x -= i0
+        idx = x.astype(np.int64)
+        np.clip(idx, 0, n - 1, out=idx)
+        return idx
+    u = draw(undirected_edges)
+    v = draw(undirected_edges)
+    relabel = rng.permutation(n).astype(np.int64)
+    return _csr_from_pairs(n, relabel[u], relabel[v])
 
 
 def chung_lu_lognormal(n: int, mean_degree: float, sigma: float, seed: int):
