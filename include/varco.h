@@ -205,6 +205,12 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
                     varco_ratio_t c, varco_key_t key, void *workspace, size_t ws_bytes,
                     uint64_t *halo_bytes, void *stream);
 
+/* Device-side status of the most recent varco_layer_fwd / varco_layer_bwd that used `workspace`:
+ * 0 = every kernel ran to completion; non-zero = a tensor-core kernel gave up on a bounded wait
+ * (its outputs are then invalid; the kernel released its resources and returned, the context stays
+ * usable).  Copies one word back on `stream` and synchronises it.  No counterpart in the paper. */
+int varco_workspace_status(const void *workspace, void *stream, int *device_status);
+
 /* ------------------------------------------------------------------------------------------
  * Per-stage device timing (no counterpart in the paper; a measurement aid).
  * When enabled, every kernel stage of the entry points above is bracketed by CUDA events on the

@@ -23,7 +23,7 @@ EXPORTS = ["varco_status_string", "varco_partition_build", "varco_partition_dest
            "varco_partition_boundary_rows", "varco_partition_counts", "varco_partition_halo", "varco_partition_perm", "varco_partition_device_bytes",
            "varco_partition_upload", "varco_workspace_bytes", "varco_kept", "varco_schedule_linear",
            "varco_compress", "varco_decompress", "varco_layer_fwd", "varco_layer_bwd", "varco_profile_enable",
-           "varco_profile_reset", "varco_profile_read", "varco_kernel_launches"]
+           "varco_profile_reset", "varco_profile_read", "varco_kernel_launches", "varco_workspace_status"]
 
 
 class Ratio(C.Structure):
@@ -82,6 +82,7 @@ def lib():
     L.varco_profile_reset.argtypes = [vp]
     L.varco_profile_read.argtypes = [vp, i64p, C.POINTER(C.c_double)]
     L.varco_kernel_launches.argtypes = [i64p]
+    L.varco_workspace_status.argtypes = [vp, vp, i32p]
     _lib = L
     return L
 
@@ -126,6 +127,13 @@ def varco_kernel_launches():
     c = C.c_int64()
     _check(lib().varco_kernel_launches(C.byref(c)), "varco_kernel_launches")
     return int(c.value)
+
+
+def varco_workspace_status(workspace):
+    """Device status word of the last layer call on this workspace (0 = ok); synchronises."""
+    v = C.c_int32()
+    _check(lib().varco_workspace_status(_ptr(workspace), _stream(), C.byref(v)), "varco_workspace_status")
+    return int(v.value)
 
 
 class Plan:

@@ -9,7 +9,7 @@
 // workspace carving shared by varco_workspace_bytes and the layer entry points
 struct varco_ws_layout {
   int64_t ld_in = 0, ld_out = 0;  // leading dimensions of the internal buffers
-  size_t packed = 0, halo = 0, dZ = 0, dAgg = 0, scratch = 0, scratch_bytes = 0, total = 0;
+  size_t status = 0, packed = 0, halo = 0, dZ = 0, dAgg = 0, scratch = 0, scratch_bytes = 0, total = 0;
 };
 varco_ws_layout varco_make_ws_layout(const varco_plan *pl, int F_in, int F_out, varco_dtype_t dt);
 size_t varco_gemm_scratch_bytes(int F_in, int F_out);
@@ -41,5 +41,15 @@ int varco_colsum(int n, int F_out, varco_dtype_t dt, const void *dZ, int64_t ldd
                  cudaStream_t st);
 int varco_relu_mask(int n, int F_out, varco_dtype_t dt, const void *Y, int64_t ldy, const void *dY, int64_t lddy,
                     void *dZ, int64_t lddz, cudaStream_t st);
+
+// gemm_tc.cu (bf16, tcgen05)
+size_t varco_tc_scratch_bytes(int F_in, int F_out);
+int varco_tc_gemm_fwd(int n, int F_in, int F_out, const void *X, int64_t ldx, const void *Agg, int64_t lda,
+                      const void *Ws, const void *Wn, const float *bias, int relu, void *Y, int64_t ldy,
+                      void *scratch, int *err, cudaStream_t st);
+int varco_tc_gemm_dx(int n, int F_in, int F_out, const void *dZ, int64_t lddz, const void *Ws, const void *Wn,
+                     void *dXs, int64_t ldxs, void *dAgg, int64_t ldagg, void *scratch, int *err, cudaStream_t st);
+int varco_tc_gemm_dw(int n, int F_in, int F_out, const void *X, int64_t ldx, const void *Agg, int64_t lda,
+                     const void *dZ, int64_t lddz, float *dWs, float *dWn, void *scratch, int *err, cudaStream_t st);
 
 #endif  // VARCO_KERNELS_H_

@@ -32,7 +32,15 @@ int check_desc(const varco_plan *pl, const varco_layer_desc_t *d) {
 
 }  // namespace
 
-size_t varco_gemm_scratch_bytes(int F_in, int F_out) { return varco_simt_dw_scratch_bytes(F_in, F_out); }
+size_t varco_gemm_scratch_bytes(int F_in, int F_out) {
+  const size_t a = varco_simt_dw_scratch_bytes(F_in, F_out), b = varco_tc_scratch_bytes(F_in, F_out);
+  return a > b ? a : b;
+}
+
+static char *ws_base(void *workspace) {
+  char *ws = static_cast<char *>(workspace);
+  return ws + ((256 - (reinterpret_cast<uintptr_t>(ws) & 255u)) & 255u);
+}
 
 extern "C" {
 
@@ -83,11 +91,12 @@ int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   if (!workspace || !aligned16(workspace)) return VARCO_INVALID_ARG;
   const varco_ws_layout L = varco_make_ws_layout(plan, F_in, F_out, dt);
   if (ws_bytes < L.total) return VARCO_WORKSPACE_TOO_SMALL;
-  char *ws = static_cast<char *>(workspace);
-  ws += (256 - (reinterpret_cast<uintptr_t>(ws) & 255u)) & 255u;
+  char *ws = ws_base(workspace);
   void *packed = ws + L.packed;
   void *Xhalo = ws + L.halo;
+  int *status = reinterpret_cast<int *>(ws + L.status);
   cudaStream_t st = (cudaStream_t)stream;
+  VARCO_CUDA_CHECK(cudaMemsetAsync(status, 0, 256, st));
   if (halo_bytes) *halo_bytes = (uint64_t)plan->H * (uint64_t)k * es;
 
   {
@@ -107,10 +116,24 @@ int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   if (rc != VARCO_OK) return rc;
   {
     StageTimer t(plan, VARCO_STAGE_GEMM_FWD, stream);
-    rc = varco_simt_gemm_fwd((int)plan->n, F_in, F_out, dt, X, desc->ld_in, Agg_saved, desc->ld_in, W_self, W_neigh,
-                             bias, desc->relu, Y, desc->ld_out, st);
+    if (dt == VARCO_BF16 && F_out <= 256)
+      rc = varco_tc_gemm_fwd((int)plan->n, F_in, F_out, X, desc->ld_in, Agg_saved, desc->ld_in, W_self, W_neigh, bias,
+                             desc->relu, Y, desc->ld_out, ws + L.scratch, status, st);
+    else
+      rc = varco_simt_gemm_fwd((int)plan->n, F_in, F_out, dt, X, desc->ld_in, Agg_saved, desc->ld_in, W_self,
+                               W_neigh, bias, desc->relu, Y, desc->ld_out, st);
   }
   return rc;
+}
+
+int varco_workspace_status(const void *workspace, void *stream, int *device_status) {
+  if (!workspace || !device_status) return VARCO_INVALID_ARG;
+  const char *ws = ws_base(const_cast<void *>(workspace));
+  int v = 0;
+  VARCO_CUDA_CHECK(cudaMemcpyAsync(&v, ws, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+  VARCO_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream));
+  *device_status = v;
+  return VARCO_OK;
 }
 
 int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, const void *X, const void *Y,
@@ -136,8 +159,10 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   if (!workspace || !aligned16(workspace)) return VARCO_INVALID_ARG;
   const varco_ws_layout L = varco_make_ws_layout(plan, F_in, F_out, dt);
   if (ws_bytes < L.total) return VARCO_WORKSPACE_TOO_SMALL;
-  char *ws = static_cast<char *>(workspace);
-  ws += (256 - (reinterpret_cast<uintptr_t>(ws) & 255u)) & 255u;
+  char *ws = ws_base(workspace);
+  int *status = reinterpret_cast<int *>(ws + L.status);
+  VARCO_CUDA_CHECK(cudaMemsetAsync(status, 0, 256, (cudaStream_t)stream));
+  const bool tc = dt == VARCO_BF16 && F_out <= 256 && (sage ? 2 : 1) * ((F_in + 127) / 128) <= 8;
   void *packed = ws + L.packed;
   void *Ghalo = ws + L.halo;
   void *dZbuf = ws + L.dZ;
@@ -157,16 +182,26 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   }
   {
     StageTimer t(plan, VARCO_STAGE_GEMM_DW, stream);
-    rc = varco_simt_gemm_dw(n, F_in, F_out, dt, Agg_saved, desc->ld_in, dZ, lddz, dW_neigh, scratch, st);
-    if (rc == VARCO_OK && sage)
-      rc = varco_simt_gemm_dw(n, F_in, F_out, dt, X, desc->ld_in, dZ, lddz, dW_self, scratch, st);
+    if (tc) {
+      rc = varco_tc_gemm_dw(n, F_in, F_out, X, desc->ld_in, Agg_saved, desc->ld_in, dZ, lddz, dW_self, dW_neigh,
+                            scratch, status, st);
+    } else {
+      rc = varco_simt_gemm_dw(n, F_in, F_out, dt, Agg_saved, desc->ld_in, dZ, lddz, dW_neigh, scratch, st);
+      if (rc == VARCO_OK && sage)
+        rc = varco_simt_gemm_dw(n, F_in, F_out, dt, X, desc->ld_in, dZ, lddz, dW_self, scratch, st);
+    }
     if (rc == VARCO_OK && dbias) rc = varco_colsum(n, F_out, dt, dZ, lddz, dbias, scratch, st);
   }
   if (rc != VARCO_OK) return rc;
   {
     StageTimer t(plan, VARCO_STAGE_GEMM_DX, stream);
-    rc = varco_simt_gemm_dx(n, F_in, F_out, dt, dZ, lddz, W_neigh, dAgg, L.ld_in, st);
-    if (rc == VARCO_OK && sage) rc = varco_simt_gemm_dx(n, F_in, F_out, dt, dZ, lddz, W_self, dX, desc->ld_in, st);
+    if (tc) {
+      rc = varco_tc_gemm_dx(n, F_in, F_out, dZ, lddz, W_self, W_neigh, dX, desc->ld_in, dAgg, L.ld_in, scratch, status,
+                            st);
+    } else {
+      rc = varco_simt_gemm_dx(n, F_in, F_out, dt, dZ, lddz, W_neigh, dAgg, L.ld_in, st);
+      if (rc == VARCO_OK && sage) rc = varco_simt_gemm_dx(n, F_in, F_out, dt, dZ, lddz, W_self, dX, desc->ld_in, st);
+    }
   }
   if (rc != VARCO_OK) return rc;
   {

@@ -208,6 +208,7 @@ varco_ws_layout varco_make_ws_layout(const varco_plan *pl, int F_in, int F_out, 
     off += aligned(b);
     return o;
   };
+  L.status = take(256);                             // device status word of the last layer call
   L.packed = take((size_t)pl->H * F_in * es);
   L.halo = take((size_t)pl->H * L.ld_in * es);      // forward: decompressed rows; backward: slot gradients
   L.dZ = take((size_t)pl->n * L.ld_out * es);

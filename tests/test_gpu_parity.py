@@ -88,6 +88,7 @@ def test_layer_forward_and_backward(orc, cases, name, scale, layer, ratio):
     Y, Agg, hb = vb.varco_layer_fwd(case.plan, Xd, Wsd, Wnd, bd, relu, ratio, key, case.ws, F_in=F_in)
     Yr, Aggr, hbr = case.g.layer_fwd(X, Ws, Wn, b, relu, ratio, key, elem_bytes=case.es)
     assert hb == hbr == case.g.H_total * orc.kept(F_in, ratio) * case.es
+    assert vb.varco_workspace_status(case.ws) == 0
     tol = TOL[dt]
     assert rel_err(to_host_rows(Agg, case.perm, F_in), Aggr) <= tol
     assert rel_err(to_host_rows(Y, case.perm, F_out), Yr) <= tol
@@ -105,6 +106,7 @@ def test_layer_forward_and_backward(orc, cases, name, scale, layer, ratio):
                                                F_in=F_in)
     rX, rWs, rWn, rb, hb2r = case.g.layer_bwd(X, Y_shared, Ws, Wn, dY, relu, ratio, key, elem_bytes=case.es)
     assert hb2 == hb2r == hb
+    assert vb.varco_workspace_status(case.ws) == 0
     assert rel_err(to_host_rows(dX, case.perm, F_in), rX) <= tol
     assert rel_err(host64(dWn), rWn) <= tol
     assert rel_err(host64(db), rb) <= tol
