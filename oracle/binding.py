@@ -41,6 +41,7 @@ class Oracle:
         L.orc_mix64.argtypes = [C.c_uint64]
         L.orc_perm_indices.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint64, C.c_int, C.c_int,
                                        C.POINTER(C.c_int32)]
+        L.orc_wire_positions.argtypes = L.orc_perm_indices.argtypes
         L.orc_perm_inverse.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint64, C.c_int, C.c_int]
         L.orc_round_keys.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint64, C.c_int, C.POINTER(C.c_uint32)]
         L.orc_kept.argtypes = [C.c_int, C.c_uint64, C.c_uint64]
@@ -80,6 +81,13 @@ class Oracle:
         rc = self.lib.orc_perm_indices(seed, epoch, layer, node, F, k, _p(out, C.c_int32))
         if rc != 0:
             raise ValueError("bad permutation arguments")
+        return out
+
+    def wire_positions(self, seed, epoch, layer, node, F, k):
+        out = np.empty(k, dtype=np.int32)
+        rc = self.lib.orc_wire_positions(seed, epoch, layer, node, F, k, _p(out, C.c_int32))
+        if rc != 0:
+            raise ValueError("bad arguments")
         return out
 
     def perm_inverse(self, seed, epoch, layer, node, F, c):

@@ -169,14 +169,21 @@ struct LayerArgs {
   int elem_bytes;
 };
 
-// compress one row: z[m] = x[pi(m)], m < k   (appendix "Compression Mechanism")
+// Position of the m-th value on the wire.  For k < F the kept positions are the first k images of
+// the keyed permutation, sent in that order.  At full communication (k == F) nothing is dropped
+// and the row is sent as it is: the paper's "full communication" setting involves no compressor,
+// and the order of a complete row on the wire is not observable in its terms.
+uint32_t wire_position(const KeyedPerm& kp, int m, int k) {
+  return (k == (int)kp.F) ? (uint32_t)m : kp.pi((uint32_t)m);
+}
+// compress one row: z[m] = x[position(m)], m < k   (appendix "Compression Mechanism")
 void compress_row(const KeyedPerm& kp, const double* x, int k, double* z) {
-  for (int m = 0; m < k; ++m) z[m] = x[kp.pi((uint32_t)m)];
+  for (int m = 0; m < k; ++m) z[m] = x[wire_position(kp, m, k)];
 }
 // decompress one row: values put back in place, zero everywhere else
 void decompress_row(const KeyedPerm& kp, const double* z, int k, int F, double* xt) {
   for (int c = 0; c < F; ++c) xt[c] = 0.0;
-  for (int m = 0; m < k; ++m) xt[kp.pi((uint32_t)m)] = z[m];
+  for (int m = 0; m < k; ++m) xt[wire_position(kp, m, k)] = z[m];
 }
 
 // Steps 2-3 of Algorithm 1 for one layer: every worker p compresses its
@@ -292,6 +299,13 @@ int orc_perm_indices(uint64_t seed, uint32_t epoch, uint32_t layer, uint64_t nod
   if (F < 1 || k < 0 || k > F) return -1;
   KeyedPerm kp(seed, epoch, layer, node, F);
   for (int m = 0; m < k; ++m) idx[m] = (int32_t)kp.pi((uint32_t)m);
+  return 0;
+}
+// positions of the k values of a row in the order they are sent
+int orc_wire_positions(uint64_t seed, uint32_t epoch, uint32_t layer, uint64_t node, int F, int k, int32_t* idx) {
+  if (F < 1 || k < 0 || k > F) return -1;
+  KeyedPerm kp(seed, epoch, layer, node, F);
+  for (int m = 0; m < k; ++m) idx[m] = (int32_t)wire_position(kp, m, k);
   return 0;
 }
 int orc_perm_inverse(uint64_t seed, uint32_t epoch, uint32_t layer, uint64_t node, int F, int c) {

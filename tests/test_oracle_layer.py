@@ -81,7 +81,11 @@ def test_decompress_of_compress_is_the_masked_row_bit_exact(orc):
         for q in range(wl.parts):
             for p in range(wl.parts):
                 for r, j in enumerate(g.halo(p, q)):
-                    idx = orc.perm_indices(*KEY, int(j), F, k)
+                    idx = orc.wire_positions(*KEY, int(j), F, k)
+                    if k < F:       # kept positions: the first k images of the keyed permutation
+                        assert np.array_equal(idx, orc.perm_indices(*KEY, int(j), F, k))
+                    else:           # full communication: the row as it is
+                        assert np.array_equal(idx, np.arange(F))
                     assert np.array_equal(packed[pos[(p, q)] + r], X[j, idx])
                     want = np.zeros(F)
                     want[idx] = X[j, idx]
