@@ -5,116 +5,213 @@
 // compressor keeps k = ceil(F / c) values of a row at keyed pseudo-random positions and the
 // decoder puts them back in place with zeros elsewhere (Definition 1; appendix "Compression
 // Mechanism").  The backward pass returns the halo-row gradients through the same compressor.
+// At full communication (k == F) nothing is dropped and rows travel in their natural order, so
+// the exchange is a plain row copy.
 //
-// All four kernels are pure data movement (bit-exact) plus the integer permutation, one warp per
-// row: the row is staged in shared memory with 128-bit accesses, permuted there, and the packed
-// side is written/read as contiguous k-element rows.
+// The kernels are data movement (bit-exact) plus the integer permutation.  A group of G lanes
+// (8, 16 or 32, by row width) owns one row, so that a warp keeps several rows in flight; rows are
+// staged in shared memory with 128-bit accesses and permuted there; packed rows are read and
+// written with 128-bit accesses whenever their stride allows it.
+//
+// Packed buffers come in two orders.  The layer path writes a copy straight to the position of
+// its halo slot at the receiver ("receive order": destination, owner, id), which folds the
+// exchange step into the write address.  The stand-alone compress / decompress entry points use
+// the sender's order (owner, destination, id) on the packed side.
 #include "device_common.cuh"
+#include "kernels.h"
 
 namespace {
 
-constexpr int kWarp = 32;
-
 template <typename E> struct VecOf { static constexpr int kVec = 16 / (int)sizeof(E); };
 
-__device__ __forceinline__ uint4 ld_nc(const uint4 *p) { return __ldg(p); }
+template <int G> __device__ __forceinline__ unsigned group_mask() {
+  if (G == 32) return 0xFFFFFFFFu;
+  const unsigned lane = threadIdx.x & 31u;
+  return ((1u << G) - 1u) << (lane & ~(unsigned)(G - 1));
+}
+
+// Round keys of one row, computed by six lanes of the group and shared by shuffle.
+template <int G>
+__device__ __forceinline__ void init_perm(vperm::RowPerm &pm, uint64_t lkey, uint32_t node, uint32_t F, int h, int gl,
+                                          unsigned gmask) {
+  const uint64_t a = vperm::mix(lkey + (uint64_t)node);
+  uint32_t mine = 0;
+  if (gl < 6) mine = (uint32_t)(vperm::mix(a + (uint64_t)(gl + 1) * vperm::kPhi64) >> 32) * vperm::kGold32;
+#pragma unroll
+  for (int i = 0; i < 6; ++i) pm.rkg[i] = __shfl_sync(gmask, mine, i, G);
+  pm.F = F;
+  pm.h = h;
+}
+
+__device__ __forceinline__ uint32_t wire_pos(const vperm::RowPerm &pm, int m, bool identity) {
+  return identity ? (uint32_t)m : pm.pi((uint32_t)m);
+}
 
 // ------------------------------------------------------------------------------------------
-// Forward, sender side.  One warp per UNIQUE boundary row: the row is read once, its k kept
-// values are selected once and written to the send segment of every destination partition.
-template <typename E>
+// Full communication, sender side: copy every unique boundary row into the halo slot of every
+// partition that uses it.  Works on 16-byte chunks, any element type.
+template <int G>
+__global__ void __launch_bounds__(256) gather_copy_kernel(const uint4 *__restrict__ X, int64_t ldx4, int nv,
+                                                          const int32_t *__restrict__ brow,
+                                                          const int32_t *__restrict__ brow_ptr,
+                                                          const int32_t *__restrict__ brow_slot, int nb,
+                                                          uint4 *__restrict__ Xhalo, int64_t ldh4) {
+  const int b = (blockIdx.x * blockDim.x + threadIdx.x) / G;
+  const int gl = threadIdx.x % G;
+  if (b >= nb) return;
+  const int r = brow[b];
+  const int s0 = brow_ptr[b], s1 = brow_ptr[b + 1];
+  const uint4 *src = X + (int64_t)r * ldx4;
+  for (int v0 = 0; v0 < nv; v0 += 4 * G) {
+    uint4 val[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int v = v0 + u * G + gl;
+      val[u] = v < nv ? __ldg(src + v) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    for (int s = s0; s < s1; ++s) {
+      uint4 *dst = Xhalo + (int64_t)brow_slot[s] * ldh4;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int v = v0 + u * G + gl;
+        if (v < nv) dst[v] = val[u];
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Sender side, general k.  One group per unique boundary row: the row is read once, its k kept
+// values are selected once and written to the copy of every destination partition.
+template <typename E, int G>
 __global__ void __launch_bounds__(256) compress_rows_kernel(const E *__restrict__ X, int64_t ld, int F, int k, int h,
                                                             uint64_t lkey, const int32_t *__restrict__ brow,
                                                             const int32_t *__restrict__ brow_ptr,
                                                             const int32_t *__restrict__ brow_slot,
                                                             const int32_t *__restrict__ slot_sendpos,
                                                             const int32_t *__restrict__ row_gid, int nb,
-                                                            E *__restrict__ packed) {
+                                                            E *__restrict__ packed, int64_t kstride) {
   extern __shared__ uint4 smem_u4[];
   constexpr int V = VecOf<E>::kVec;
-  const int nv = (F + V - 1) / V;
-  const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
-  const int wpb = blockDim.x / kWarp;
-  const int b = blockIdx.x * wpb + warp;
+  const int nv = (F + V - 1) / V;      // chunks of a row
+  const int kv = (k + V - 1) / V;      // chunks of a packed row
+  const int grp = threadIdx.x / G, gl = threadIdx.x % G;
+  const int b = blockIdx.x * (blockDim.x / G) + grp;
   if (b >= nb) return;
-  uint4 *srow4 = smem_u4 + (size_t)warp * nv;
+  const unsigned gmask = group_mask<G>();
+  uint4 *srow4 = smem_u4 + (size_t)grp * (nv + kv);
+  uint4 *zrow4 = srow4 + nv;
   const E *srow = reinterpret_cast<const E *>(srow4);
+  E *zrow = reinterpret_cast<E *>(zrow4);
   const int r = brow[b];
-  const uint4 *src = reinterpret_cast<const uint4 *>(X + (int64_t)r * ld);
-  for (int v = lane; v < nv; v += kWarp) srow4[v] = ld_nc(src + v);
-  vperm::RowPerm pm;
-  pm.init(lkey, (uint32_t)row_gid[r], (uint32_t)F, h);
   const int s0 = brow_ptr[b], s1 = brow_ptr[b + 1];
-  __syncwarp();
-  for (int m = lane; m < k; m += kWarp) {
-    const E v = srow[pm.pi((uint32_t)m)];
-    for (int s = s0; s < s1; ++s) {
-      const int64_t pos = slot_sendpos[brow_slot[s]];
-      packed[pos * k + m] = v;
+  const uint4 *src = reinterpret_cast<const uint4 *>(X + (int64_t)r * ld);
+  for (int v = gl; v < nv; v += G) srow4[v] = __ldg(src + v);
+  vperm::RowPerm pm;
+  init_perm<G>(pm, lkey, (uint32_t)row_gid[r], (uint32_t)F, h, gl, gmask);
+  const bool identity = k == F;
+  __syncwarp(gmask);
+  for (int m = gl; m < kv * V; m += G) zrow[m] = m < k ? srow[wire_pos(pm, m, identity)] : (E)0;
+  __syncwarp(gmask);
+  const bool vec = ((kstride * (int64_t)sizeof(E)) & 15) == 0;
+  for (int s = s0; s < s1; ++s) {
+    const int slot = brow_slot[s];
+    const int64_t pos = slot_sendpos ? (int64_t)slot_sendpos[slot] : (int64_t)slot;
+    E *dst = packed + pos * kstride;
+    if (vec) {
+      uint4 *dst4 = reinterpret_cast<uint4 *>(dst);
+      for (int v = gl; v < kv; v += G) dst4[v] = zrow4[v];
+    } else {
+      for (int m = gl; m < k; m += G) dst[m] = zrow[m];
     }
   }
 }
 
 // ------------------------------------------------------------------------------------------
-// Forward, receiver side.  One warp per halo slot: the k received values are put back at
-// their positions in a zeroed row, which is then written out densely.
-template <typename E>
-__global__ void __launch_bounds__(256) decompress_slots_kernel(const E *__restrict__ packed, int F, int k, int h,
-                                                               uint64_t lkey, const int32_t *__restrict__ slot_gid,
+// Receiver side.  One group per halo slot: the k received values are put back at their
+// positions in a zeroed row, which is then written out densely.
+template <typename E, int G>
+__global__ void __launch_bounds__(256) decompress_slots_kernel(const E *__restrict__ packed, int64_t kstride, int F,
+                                                               int k, int h, uint64_t lkey,
+                                                               const int32_t *__restrict__ slot_gid,
                                                                const int32_t *__restrict__ slot_sendpos, int H,
                                                                E *__restrict__ Xhalo, int64_t ld) {
   extern __shared__ uint4 smem_u4[];
   constexpr int V = VecOf<E>::kVec;
   const int nv = (F + V - 1) / V;
-  const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
-  const int wpb = blockDim.x / kWarp;
-  const int slot = blockIdx.x * wpb + warp;
+  const int kv = (k + V - 1) / V;
+  const int grp = threadIdx.x / G, gl = threadIdx.x % G;
+  const int slot = blockIdx.x * (blockDim.x / G) + grp;
   if (slot >= H) return;
-  uint4 *srow4 = smem_u4 + (size_t)warp * nv;
+  const unsigned gmask = group_mask<G>();
+  uint4 *srow4 = smem_u4 + (size_t)grp * (nv + kv);
+  uint4 *zrow4 = srow4 + nv;
   E *srow = reinterpret_cast<E *>(srow4);
-  for (int v = lane; v < nv; v += kWarp) srow4[v] = make_uint4(0u, 0u, 0u, 0u);
+  E *zrow = reinterpret_cast<E *>(zrow4);
+  const int64_t pos = slot_sendpos ? (int64_t)slot_sendpos[slot] : (int64_t)slot;
+  const E *z = packed + pos * kstride;
+  const bool vec = ((kstride * (int64_t)sizeof(E)) & 15) == 0;
+  if (vec) {
+    const uint4 *z4 = reinterpret_cast<const uint4 *>(z);
+    for (int v = gl; v < kv; v += G) zrow4[v] = __ldg(z4 + v);
+  } else {
+    for (int m = gl; m < k; m += G) zrow[m] = z[m];
+  }
+  for (int v = gl; v < nv; v += G) srow4[v] = make_uint4(0u, 0u, 0u, 0u);
   vperm::RowPerm pm;
-  pm.init(lkey, (uint32_t)slot_gid[slot], (uint32_t)F, h);
-  const E *z = packed + (int64_t)slot_sendpos[slot] * k;
-  __syncwarp();
-  for (int m = lane; m < k; m += kWarp) srow[pm.pi((uint32_t)m)] = z[m];
-  __syncwarp();
+  init_perm<G>(pm, lkey, (uint32_t)slot_gid[slot], (uint32_t)F, h, gl, gmask);
+  const bool identity = k == F;
+  __syncwarp(gmask);
+  for (int m = gl; m < k; m += G) srow[wire_pos(pm, m, identity)] = zrow[m];
+  __syncwarp(gmask);
   uint4 *dst = reinterpret_cast<uint4 *>(Xhalo + (int64_t)slot * ld);
-  for (int v = lane; v < nv; v += kWarp) dst[v] = srow4[v];
+  for (int v = gl; v < nv; v += G) dst[v] = srow4[v];
 }
 
 // ------------------------------------------------------------------------------------------
-// Backward, receiver side (now the sender of gradients).  One warp per halo slot: the slot's
-// gradient row is compressed with the forward's permutation; packed rows are in slot order.
-template <typename E>
-__global__ void __launch_bounds__(256) compress_slots_kernel(const E *__restrict__ G, int64_t ld, int F, int k, int h,
+// Backward, receiver side (now the sender of gradients), k < F.  One group per halo slot: the
+// slot's gradient row is compressed with the forward's permutation; packed rows in slot order.
+template <typename E, int G>
+__global__ void __launch_bounds__(256) compress_slots_kernel(const E *__restrict__ Gh, int64_t ld, int F, int k, int h,
                                                              uint64_t lkey, const int32_t *__restrict__ slot_gid,
-                                                             int H, E *__restrict__ packed) {
+                                                             int H, E *__restrict__ packed, int64_t kstride) {
   extern __shared__ uint4 smem_u4[];
   constexpr int V = VecOf<E>::kVec;
   const int nv = (F + V - 1) / V;
-  const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
-  const int wpb = blockDim.x / kWarp;
-  const int slot = blockIdx.x * wpb + warp;
+  const int kv = (k + V - 1) / V;
+  const int grp = threadIdx.x / G, gl = threadIdx.x % G;
+  const int slot = blockIdx.x * (blockDim.x / G) + grp;
   if (slot >= H) return;
-  uint4 *srow4 = smem_u4 + (size_t)warp * nv;
+  const unsigned gmask = group_mask<G>();
+  uint4 *srow4 = smem_u4 + (size_t)grp * (nv + kv);
+  uint4 *zrow4 = srow4 + nv;
   const E *srow = reinterpret_cast<const E *>(srow4);
-  const uint4 *src = reinterpret_cast<const uint4 *>(G + (int64_t)slot * ld);
-  for (int v = lane; v < nv; v += kWarp) srow4[v] = ld_nc(src + v);
+  E *zrow = reinterpret_cast<E *>(zrow4);
+  const uint4 *src = reinterpret_cast<const uint4 *>(Gh + (int64_t)slot * ld);
+  for (int v = gl; v < nv; v += G) srow4[v] = __ldg(src + v);
   vperm::RowPerm pm;
-  pm.init(lkey, (uint32_t)slot_gid[slot], (uint32_t)F, h);
-  E *z = packed + (int64_t)slot * k;
-  __syncwarp();
-  for (int m = lane; m < k; m += kWarp) z[m] = srow[pm.pi((uint32_t)m)];
+  init_perm<G>(pm, lkey, (uint32_t)slot_gid[slot], (uint32_t)F, h, gl, gmask);
+  const bool identity = k == F;
+  __syncwarp(gmask);
+  for (int m = gl; m < kv * V; m += G) zrow[m] = m < k ? srow[wire_pos(pm, m, identity)] : (E)0;
+  __syncwarp(gmask);
+  E *dst = packed + (int64_t)slot * kstride;
+  if (((kstride * (int64_t)sizeof(E)) & 15) == 0) {
+    uint4 *dst4 = reinterpret_cast<uint4 *>(dst);
+    for (int v = gl; v < kv; v += G) dst4[v] = zrow4[v];
+  } else {
+    for (int m = gl; m < k; m += G) dst[m] = zrow[m];
+  }
 }
 
 // ------------------------------------------------------------------------------------------
-// Backward, owner side.  One warp per unique boundary row: the packed gradients returned by
-// every destination partition are summed in ascending destination order and added to the
-// owner's gradient row at the kept positions.  No atomics: the result is reproducible.
-template <typename T>
-__global__ void __launch_bounds__(256) scatter_add_rows_kernel(const T *__restrict__ packed, int F, int k, int h,
-                                                               uint64_t lkey, const int32_t *__restrict__ brow,
+// Backward, owner side, k < F.  One group per unique boundary row: the packed gradients
+// returned by every destination partition are summed in ascending destination order and added
+// to the owner's gradient row at the kept positions.  No atomics: the result is reproducible.
+template <typename T, int G>
+__global__ void __launch_bounds__(256) scatter_add_rows_kernel(const T *__restrict__ packed, int64_t kstride, int F,
+                                                               int k, int h, uint64_t lkey,
+                                                               const int32_t *__restrict__ brow,
                                                                const int32_t *__restrict__ brow_ptr,
                                                                const int32_t *__restrict__ brow_slot,
                                                                const int32_t *__restrict__ row_gid, int nb,
@@ -122,30 +219,30 @@ __global__ void __launch_bounds__(256) scatter_add_rows_kernel(const T *__restri
   extern __shared__ uint4 smem_u4[];
   constexpr int V = ElemTraits<T>::kVec;
   const int nv = (F + V - 1) / V;
-  const int warp = threadIdx.x / kWarp, lane = threadIdx.x % kWarp;
-  const int wpb = blockDim.x / kWarp;
-  const int b = blockIdx.x * wpb + warp;
+  const int grp = threadIdx.x / G, gl = threadIdx.x % G;
+  const int b = blockIdx.x * (blockDim.x / G) + grp;
   if (b >= nb) return;
-  float *srow = reinterpret_cast<float *>(smem_u4) + (size_t)warp * nv * V;
+  const unsigned gmask = group_mask<G>();
+  float *srow = reinterpret_cast<float *>(smem_u4) + (size_t)grp * nv * V;
   const int r = brow[b];
+  const int s0 = brow_ptr[b], s1 = brow_ptr[b + 1];
   uint4 *row4 = reinterpret_cast<uint4 *>(dX + (int64_t)r * ld);
-  for (int v = lane; v < nv; v += kWarp) {
+  for (int v = gl; v < nv; v += G) {
     float f[V];
     unpack16(row4[v], f, T());
 #pragma unroll
     for (int i = 0; i < V; ++i) srow[v * V + i] = f[i];
   }
   vperm::RowPerm pm;
-  pm.init(lkey, (uint32_t)row_gid[r], (uint32_t)F, h);
-  const int s0 = brow_ptr[b], s1 = brow_ptr[b + 1];
-  __syncwarp();
-  for (int m = lane; m < k; m += kWarp) {
+  init_perm<G>(pm, lkey, (uint32_t)row_gid[r], (uint32_t)F, h, gl, gmask);
+  __syncwarp(gmask);
+  for (int m = gl; m < k; m += G) {
     float sum = 0.f;
-    for (int s = s0; s < s1; ++s) sum += ElemTraits<T>::to_f(packed[(int64_t)brow_slot[s] * k + m]);
+    for (int s = s0; s < s1; ++s) sum += ElemTraits<T>::to_f(packed[(int64_t)brow_slot[s] * kstride + m]);
     srow[pm.pi((uint32_t)m)] += sum;
   }
-  __syncwarp();
-  for (int v = lane; v < nv; v += kWarp) {
+  __syncwarp(gmask);
+  for (int v = gl; v < nv; v += G) {
     float f[V];
 #pragma unroll
     for (int i = 0; i < V; ++i) f[i] = srow[v * V + i];
@@ -153,98 +250,191 @@ __global__ void __launch_bounds__(256) scatter_add_rows_kernel(const T *__restri
   }
 }
 
-int warps_per_block(size_t row_bytes) {
-  int w = (int)(48 * 1024 / row_bytes);
-  if (w >= 8) return 8;
-  if (w >= 4) return 4;
-  if (w >= 2) return 2;
-  return 1;
+// Backward, owner side, full communication: the slot gradient rows are dense; add them to the
+// owner's row in ascending destination order.
+template <typename T, int G>
+__global__ void __launch_bounds__(256) add_dense_rows_kernel(const T *__restrict__ Gh, int64_t ldg, int nv,
+                                                             const int32_t *__restrict__ brow,
+                                                             const int32_t *__restrict__ brow_ptr,
+                                                             const int32_t *__restrict__ brow_slot, int nb,
+                                                             T *__restrict__ dX, int64_t ld) {
+  constexpr int V = ElemTraits<T>::kVec;
+  const int b = (blockIdx.x * blockDim.x + threadIdx.x) / G;
+  const int gl = threadIdx.x % G;
+  if (b >= nb) return;
+  const int r = brow[b];
+  const int s0 = brow_ptr[b], s1 = brow_ptr[b + 1];
+  uint4 *row4 = reinterpret_cast<uint4 *>(dX + (int64_t)r * ld);
+  for (int v = gl; v < nv; v += G) {
+    float acc[V];
+    unpack16(row4[v], acc, T());
+    int s = s0;
+    for (; s + 1 < s1; s += 2) {
+      const uint4 a = __ldg(reinterpret_cast<const uint4 *>(Gh + (int64_t)brow_slot[s] * ldg) + v);
+      const uint4 c = __ldg(reinterpret_cast<const uint4 *>(Gh + (int64_t)brow_slot[s + 1] * ldg) + v);
+      float fa[V], fc[V];
+      unpack16(a, fa, T());
+      unpack16(c, fc, T());
+#pragma unroll
+      for (int i = 0; i < V; ++i) acc[i] = (acc[i] + fa[i]) + fc[i];
+    }
+    if (s < s1) {
+      float fa[V];
+      unpack16(__ldg(reinterpret_cast<const uint4 *>(Gh + (int64_t)brow_slot[s] * ldg) + v), fa, T());
+#pragma unroll
+      for (int i = 0; i < V; ++i) acc[i] += fa[i];
+    }
+    row4[v] = pack16(acc, T());
+  }
 }
+
+int group_size(int nv) { return nv <= 32 ? 8 : (nv <= 64 ? 16 : 32); }
+
+struct HaloLaunch {
+  int G, threads;
+  unsigned blocks;
+  size_t smem;
+};
+// rows -> launch shape; `row_smem` bytes of shared memory per row
+HaloLaunch shape(int64_t rows, int nv, size_t row_smem) {
+  HaloLaunch L;
+  L.G = group_size(nv);
+  L.threads = 256;
+  while (L.threads > L.G && (size_t)(L.threads / L.G) * row_smem > 48 * 1024) L.threads /= 2;
+  const int per_block = L.threads / L.G;
+  L.blocks = (unsigned)((rows + per_block - 1) / per_block);
+  L.smem = (size_t)per_block * row_smem;
+  return L;
+}
+
+#define VARCO_DISPATCH_G(L, CALL)   \
+  do {                              \
+    if ((L).G == 8) {               \
+      constexpr int G = 8;          \
+      CALL;                         \
+    } else if ((L).G == 16) {       \
+      constexpr int G = 16;         \
+      CALL;                         \
+    } else {                        \
+      constexpr int G = 32;         \
+      CALL;                         \
+    }                               \
+  } while (0)
 
 }  // namespace
 
 // ------------------------------------------------------------------------------------------ launchers
-int varco_launch_compress_rows(const varco_plan *pl, const void *X, int64_t ld, int F, int k, varco_dtype_t dt,
-                               varco_key_t key, void *packed, cudaStream_t st) {
+// Full-communication exchange of the layer path: X rows -> dense halo slots.
+int varco_launch_gather_copy(const varco_plan *pl, const void *X, int64_t ld, int F, varco_dtype_t dt, void *Xhalo,
+                             int64_t ldh, cudaStream_t st) {
   if (pl->nb == 0) return VARCO_OK;
-  const int es = dt == VARCO_F32 ? 4 : 2;
-  const int V = 16 / es;
-  const size_t row_bytes = (size_t)((F + V - 1) / V) * 16;
-  const int wpb = warps_per_block(row_bytes);
-  const int h = vperm::half_bits(F);
-  const uint64_t lkey = vperm::layer_key(key);
-  dim3 grid((unsigned)((pl->nb + wpb - 1) / wpb)), block(wpb * 32);
-  if (dt == VARCO_F32)
-    compress_rows_kernel<uint32_t><<<grid, block, row_bytes * wpb, st>>>(
-        (const uint32_t *)X, ld, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot, pl->d.slot_sendpos,
-        pl->d.row_gid, (int)pl->nb, (uint32_t *)packed);
-  else
-    compress_rows_kernel<uint16_t><<<grid, block, row_bytes * wpb, st>>>(
-        (const uint16_t *)X, ld, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot, pl->d.slot_sendpos,
-        pl->d.row_gid, (int)pl->nb, (uint16_t *)packed);
+  const int es = dt == VARCO_F32 ? 4 : 2, V = 16 / es;
+  const int nv = (F + V - 1) / V;
+  HaloLaunch L = shape(pl->nb, nv, 0);
+  VARCO_DISPATCH_G(L, (gather_copy_kernel<G><<<L.blocks, L.threads, 0, st>>>(
+                          (const uint4 *)X, ld / V, nv, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot, (int)pl->nb,
+                          (uint4 *)Xhalo, ldh / V)));
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
-int varco_launch_decompress_slots(const varco_plan *pl, const void *packed, int F, int k, varco_dtype_t dt,
-                                  varco_key_t key, void *Xhalo, int64_t ld, cudaStream_t st) {
+// send_order != 0: packed rows at the sender's positions (stand-alone entry point), else at the slot
+int varco_launch_compress_rows(const varco_plan *pl, const void *X, int64_t ld, int F, int k, varco_dtype_t dt,
+                               varco_key_t key, void *packed, int64_t kstride, int send_order, cudaStream_t st) {
+  if (pl->nb == 0) return VARCO_OK;
+  const int es = dt == VARCO_F32 ? 4 : 2, V = 16 / es;
+  const int nv = (F + V - 1) / V, kv = (k + V - 1) / V;
+  HaloLaunch L = shape(pl->nb, nv, (size_t)(nv + kv) * 16);
+  const int h = vperm::half_bits(F);
+  const uint64_t lkey = vperm::layer_key(key);
+  const int32_t *sp = send_order ? pl->d.slot_sendpos : nullptr;
+  if (dt == VARCO_F32)
+    VARCO_DISPATCH_G(L, (compress_rows_kernel<uint32_t, G><<<L.blocks, L.threads, L.smem, st>>>(
+                            (const uint32_t *)X, ld, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot, sp,
+                            pl->d.row_gid, (int)pl->nb, (uint32_t *)packed, kstride)));
+  else
+    VARCO_DISPATCH_G(L, (compress_rows_kernel<uint16_t, G><<<L.blocks, L.threads, L.smem, st>>>(
+                            (const uint16_t *)X, ld, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot, sp,
+                            pl->d.row_gid, (int)pl->nb, (uint16_t *)packed, kstride)));
+  VARCO_KERNEL_LAUNCHED();
+  return VARCO_OK;
+}
+
+int varco_launch_decompress_slots(const varco_plan *pl, const void *packed, int64_t kstride, int send_order, int F,
+                                  int k, varco_dtype_t dt, varco_key_t key, void *Xhalo, int64_t ld, cudaStream_t st) {
   if (pl->H == 0) return VARCO_OK;
-  const int es = dt == VARCO_F32 ? 4 : 2;
-  const int V = 16 / es;
-  const size_t row_bytes = (size_t)((F + V - 1) / V) * 16;
-  const int wpb = warps_per_block(row_bytes);
+  const int es = dt == VARCO_F32 ? 4 : 2, V = 16 / es;
+  const int nv = (F + V - 1) / V, kv = (k + V - 1) / V;
+  HaloLaunch L = shape(pl->H, nv, (size_t)(nv + kv) * 16);
   const int h = vperm::half_bits(F);
   const uint64_t lkey = vperm::layer_key(key);
-  dim3 grid((unsigned)((pl->H + wpb - 1) / wpb)), block(wpb * 32);
+  const int32_t *sp = send_order ? pl->d.slot_sendpos : nullptr;
   if (dt == VARCO_F32)
-    decompress_slots_kernel<uint32_t><<<grid, block, row_bytes * wpb, st>>>(
-        (const uint32_t *)packed, F, k, h, lkey, pl->d.slot_gid, pl->d.slot_sendpos, (int)pl->H, (uint32_t *)Xhalo,
-        ld);
+    VARCO_DISPATCH_G(L, (decompress_slots_kernel<uint32_t, G><<<L.blocks, L.threads, L.smem, st>>>(
+                            (const uint32_t *)packed, kstride, F, k, h, lkey, pl->d.slot_gid, sp, (int)pl->H,
+                            (uint32_t *)Xhalo, ld)));
   else
-    decompress_slots_kernel<uint16_t><<<grid, block, row_bytes * wpb, st>>>(
-        (const uint16_t *)packed, F, k, h, lkey, pl->d.slot_gid, pl->d.slot_sendpos, (int)pl->H, (uint16_t *)Xhalo,
-        ld);
+    VARCO_DISPATCH_G(L, (decompress_slots_kernel<uint16_t, G><<<L.blocks, L.threads, L.smem, st>>>(
+                            (const uint16_t *)packed, kstride, F, k, h, lkey, pl->d.slot_gid, sp, (int)pl->H,
+                            (uint16_t *)Xhalo, ld)));
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
-int varco_launch_compress_slots(const varco_plan *pl, const void *G, int64_t ld, int F, int k, varco_dtype_t dt,
-                                varco_key_t key, void *packed, cudaStream_t st) {
+int varco_launch_compress_slots(const varco_plan *pl, const void *Gh, int64_t ld, int F, int k, varco_dtype_t dt,
+                                varco_key_t key, void *packed, int64_t kstride, cudaStream_t st) {
   if (pl->H == 0) return VARCO_OK;
-  const int es = dt == VARCO_F32 ? 4 : 2;
-  const int V = 16 / es;
-  const size_t row_bytes = (size_t)((F + V - 1) / V) * 16;
-  const int wpb = warps_per_block(row_bytes);
+  const int es = dt == VARCO_F32 ? 4 : 2, V = 16 / es;
+  const int nv = (F + V - 1) / V, kv = (k + V - 1) / V;
+  HaloLaunch L = shape(pl->H, nv, (size_t)(nv + kv) * 16);
   const int h = vperm::half_bits(F);
   const uint64_t lkey = vperm::layer_key(key);
-  dim3 grid((unsigned)((pl->H + wpb - 1) / wpb)), block(wpb * 32);
   if (dt == VARCO_F32)
-    compress_slots_kernel<uint32_t><<<grid, block, row_bytes * wpb, st>>>(
-        (const uint32_t *)G, ld, F, k, h, lkey, pl->d.slot_gid, (int)pl->H, (uint32_t *)packed);
+    VARCO_DISPATCH_G(L, (compress_slots_kernel<uint32_t, G><<<L.blocks, L.threads, L.smem, st>>>(
+                            (const uint32_t *)Gh, ld, F, k, h, lkey, pl->d.slot_gid, (int)pl->H, (uint32_t *)packed,
+                            kstride)));
   else
-    compress_slots_kernel<uint16_t><<<grid, block, row_bytes * wpb, st>>>(
-        (const uint16_t *)G, ld, F, k, h, lkey, pl->d.slot_gid, (int)pl->H, (uint16_t *)packed);
+    VARCO_DISPATCH_G(L, (compress_slots_kernel<uint16_t, G><<<L.blocks, L.threads, L.smem, st>>>(
+                            (const uint16_t *)Gh, ld, F, k, h, lkey, pl->d.slot_gid, (int)pl->H, (uint16_t *)packed,
+                            kstride)));
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
-int varco_launch_scatter_add_rows(const varco_plan *pl, const void *packed, int F, int k, varco_dtype_t dt,
-                                  varco_key_t key, void *dX, int64_t ld, cudaStream_t st) {
+int varco_launch_scatter_add_rows(const varco_plan *pl, const void *packed, int64_t kstride, int F, int k,
+                                  varco_dtype_t dt, varco_key_t key, void *dX, int64_t ld, cudaStream_t st) {
   if (pl->nb == 0) return VARCO_OK;
   const int V = dt == VARCO_F32 ? 4 : 8;
-  const size_t row_bytes = (size_t)((F + V - 1) / V) * V * sizeof(float);
-  const int wpb = warps_per_block(row_bytes);
+  const int nv = (F + V - 1) / V;
+  HaloLaunch L = shape(pl->nb, nv, (size_t)nv * V * sizeof(float));
   const int h = vperm::half_bits(F);
   const uint64_t lkey = vperm::layer_key(key);
-  dim3 grid((unsigned)((pl->nb + wpb - 1) / wpb)), block(wpb * 32);
   if (dt == VARCO_F32)
-    scatter_add_rows_kernel<float><<<grid, block, row_bytes * wpb, st>>>(
-        (const float *)packed, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot, pl->d.row_gid,
-        (int)pl->nb, (float *)dX, ld);
+    VARCO_DISPATCH_G(L, (scatter_add_rows_kernel<float, G><<<L.blocks, L.threads, L.smem, st>>>(
+                            (const float *)packed, kstride, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot,
+                            pl->d.row_gid, (int)pl->nb, (float *)dX, ld)));
   else
-    scatter_add_rows_kernel<__nv_bfloat16><<<grid, block, row_bytes * wpb, st>>>(
-        (const __nv_bfloat16 *)packed, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot, pl->d.row_gid,
-        (int)pl->nb, (__nv_bfloat16 *)dX, ld);
+    VARCO_DISPATCH_G(L, (scatter_add_rows_kernel<__nv_bfloat16, G><<<L.blocks, L.threads, L.smem, st>>>(
+                            (const __nv_bfloat16 *)packed, kstride, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr,
+                            pl->d.brow_slot, pl->d.row_gid, (int)pl->nb, (__nv_bfloat16 *)dX, ld)));
+  VARCO_KERNEL_LAUNCHED();
+  return VARCO_OK;
+}
+
+int varco_launch_add_dense_rows(const varco_plan *pl, const void *Gh, int64_t ldg, int F, varco_dtype_t dt, void *dX,
+                                int64_t ld, cudaStream_t st) {
+  if (pl->nb == 0) return VARCO_OK;
+  const int V = dt == VARCO_F32 ? 4 : 8;
+  const int nv = (F + V - 1) / V;
+  HaloLaunch L = shape(pl->nb, nv, 0);
+  if (dt == VARCO_F32)
+    VARCO_DISPATCH_G(L, (add_dense_rows_kernel<float, G><<<L.blocks, L.threads, 0, st>>>(
+                            (const float *)Gh, ldg, nv, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot, (int)pl->nb,
+                            (float *)dX, ld)));
+  else
+    VARCO_DISPATCH_G(L, (add_dense_rows_kernel<__nv_bfloat16, G><<<L.blocks, L.threads, 0, st>>>(
+                            (const __nv_bfloat16 *)Gh, ldg, nv, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot,
+                            (int)pl->nb, (__nv_bfloat16 *)dX, ld)));
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }

@@ -15,14 +15,18 @@ varco_ws_layout varco_make_ws_layout(const varco_plan *pl, int F_in, int F_out, 
 size_t varco_gemm_scratch_bytes(int F_in, int F_out);
 
 // halo.cu
+int varco_launch_gather_copy(const varco_plan *pl, const void *X, int64_t ld, int F, varco_dtype_t dt, void *Xhalo,
+                             int64_t ldh, cudaStream_t st);
 int varco_launch_compress_rows(const varco_plan *pl, const void *X, int64_t ld, int F, int k, varco_dtype_t dt,
-                               varco_key_t key, void *packed, cudaStream_t st);
-int varco_launch_decompress_slots(const varco_plan *pl, const void *packed, int F, int k, varco_dtype_t dt,
-                                  varco_key_t key, void *Xhalo, int64_t ld, cudaStream_t st);
-int varco_launch_compress_slots(const varco_plan *pl, const void *G, int64_t ld, int F, int k, varco_dtype_t dt,
-                                varco_key_t key, void *packed, cudaStream_t st);
-int varco_launch_scatter_add_rows(const varco_plan *pl, const void *packed, int F, int k, varco_dtype_t dt,
-                                  varco_key_t key, void *dX, int64_t ld, cudaStream_t st);
+                               varco_key_t key, void *packed, int64_t kstride, int send_order, cudaStream_t st);
+int varco_launch_decompress_slots(const varco_plan *pl, const void *packed, int64_t kstride, int send_order, int F,
+                                  int k, varco_dtype_t dt, varco_key_t key, void *Xhalo, int64_t ld, cudaStream_t st);
+int varco_launch_compress_slots(const varco_plan *pl, const void *Gh, int64_t ld, int F, int k, varco_dtype_t dt,
+                                varco_key_t key, void *packed, int64_t kstride, cudaStream_t st);
+int varco_launch_scatter_add_rows(const varco_plan *pl, const void *packed, int64_t kstride, int F, int k,
+                                  varco_dtype_t dt, varco_key_t key, void *dX, int64_t ld, cudaStream_t st);
+int varco_launch_add_dense_rows(const varco_plan *pl, const void *Gh, int64_t ldg, int F, varco_dtype_t dt, void *dX,
+                                int64_t ld, cudaStream_t st);
 // spmm.cu
 int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, const void *Xhalo, int64_t ldh, int F,
                           varco_dtype_t dt, void *Agg, int64_t ldagg, cudaStream_t st);

@@ -56,7 +56,7 @@ int varco_compress(const varco_plan_t *plan, const void *X, int64_t ld, int32_t 
   if (!plan->uploaded) return VARCO_NOT_UPLOADED;
   if (bytes) *bytes = (uint64_t)plan->H * (uint64_t)k * (dtype == VARCO_F32 ? 4u : 2u);
   StageTimer t(plan, VARCO_STAGE_COMPRESS, stream);
-  return varco_launch_compress_rows(plan, X, ld, F, k, dtype, key, packed, (cudaStream_t)stream);
+  return varco_launch_compress_rows(plan, X, ld, F, k, dtype, key, packed, k, 1, (cudaStream_t)stream);
 }
 
 int varco_decompress(const varco_plan_t *plan, const void *packed, int32_t F, varco_dtype_t dtype, varco_ratio_t c,
@@ -69,7 +69,7 @@ int varco_decompress(const varco_plan_t *plan, const void *packed, int32_t F, va
   if (plan->H > 0 && (!packed || check_matrix(Xhalo, ld, F, V) != VARCO_OK)) return VARCO_INVALID_ARG;
   if (!plan->uploaded) return VARCO_NOT_UPLOADED;
   StageTimer t(plan, VARCO_STAGE_DECOMPRESS, stream);
-  return varco_launch_decompress_slots(plan, packed, F, k, dtype, key, Xhalo, ld, (cudaStream_t)stream);
+  return varco_launch_decompress_slots(plan, packed, k, 1, F, k, dtype, key, Xhalo, ld, (cudaStream_t)stream);
 }
 
 int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, const void *X, const void *W_self,
@@ -99,14 +99,21 @@ int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   VARCO_CUDA_CHECK(cudaMemsetAsync(status, 0, 256, st));
   if (halo_bytes) *halo_bytes = (uint64_t)plan->H * (uint64_t)k * es;
 
-  {
+  // Exchange.  The copy of a boundary row goes straight to the position of its halo slot at the
+  // receiver, so "send buffer -> receive buffer" is folded into the write address.  At full
+  // communication the row travels whole and in order: one gather-copy fills the halo slots.
+  const int64_t kstride = round_up64(k, V);
+  if (k == F_in) {
     StageTimer t(plan, VARCO_STAGE_COMPRESS, stream);
-    rc = varco_launch_compress_rows(plan, X, desc->ld_in, F_in, k, dt, key, packed, st);
-  }
-  if (rc != VARCO_OK) return rc;
-  {
+    rc = varco_launch_gather_copy(plan, X, desc->ld_in, F_in, dt, Xhalo, L.ld_in, st);
+  } else {
+    {
+      StageTimer t(plan, VARCO_STAGE_COMPRESS, stream);
+      rc = varco_launch_compress_rows(plan, X, desc->ld_in, F_in, k, dt, key, packed, kstride, 0, st);
+    }
+    if (rc != VARCO_OK) return rc;
     StageTimer t(plan, VARCO_STAGE_DECOMPRESS, stream);
-    rc = varco_launch_decompress_slots(plan, packed, F_in, k, dt, key, Xhalo, L.ld_in, st);
+    rc = varco_launch_decompress_slots(plan, packed, kstride, 0, F_in, k, dt, key, Xhalo, L.ld_in, st);
   }
   if (rc != VARCO_OK) return rc;
   {
@@ -209,14 +216,21 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
     rc = varco_launch_spmm_bwd(plan, dAgg, L.ld_in, F_in, dt, dX, desc->ld_in, sage ? 1 : 0, Ghalo, L.ld_in, st);
   }
   if (rc != VARCO_OK) return rc;
+  // Return of the halo-slot gradients to the owners.  At full communication the slot rows are
+  // the messages; otherwise they are compressed with the forward's key first.
+  if (k == F_in) {
+    StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
+    return varco_launch_add_dense_rows(plan, Ghalo, L.ld_in, F_in, dt, dX, desc->ld_in, st);
+  }
+  const int64_t kstride = round_up64(k, V);
   {
     StageTimer t(plan, VARCO_STAGE_COMPRESS_BWD, stream);
-    rc = varco_launch_compress_slots(plan, Ghalo, L.ld_in, F_in, k, dt, key, packed, st);
+    rc = varco_launch_compress_slots(plan, Ghalo, L.ld_in, F_in, k, dt, key, packed, kstride, st);
   }
   if (rc != VARCO_OK) return rc;
   {
     StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
-    rc = varco_launch_scatter_add_rows(plan, packed, F_in, k, dt, key, dX, desc->ld_in, st);
+    rc = varco_launch_scatter_add_rows(plan, packed, kstride, F_in, k, dt, key, dX, desc->ld_in, st);
   }
   return rc;
 }

@@ -209,7 +209,7 @@ varco_ws_layout varco_make_ws_layout(const varco_plan *pl, int F_in, int F_out, 
     return o;
   };
   L.status = take(256);                             // device status word of the last layer call
-  L.packed = take((size_t)pl->H * F_in * es);
+  L.packed = take((size_t)pl->H * L.ld_in * es);    // packed rows, stride rounded up to 16 bytes
   L.halo = take((size_t)pl->H * L.ld_in * es);      // forward: decompressed rows; backward: slot gradients
   L.dZ = take((size_t)pl->n * L.ld_out * es);
   L.dAgg = take((size_t)pl->n * L.ld_in * es);
