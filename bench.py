@@ -300,6 +300,10 @@ def run_ours(args):
     ratio = parse_ratio(args.ratio)
     t0 = time.time()
     wl = synth.make_workload(args.workload, args.scale)
+    if args.parts:
+        wl.part = synth.partition_bfs_ranges(wl.row_ptr, wl.col, args.parts, wl.seed + 1)
+        wl.parts = args.parts
+        wl.note += " (repartitioned into %d BFS ranges)" % args.parts
     gen_s = time.time() - t0
     model = DeviceModel(wl, device)
     L = model.L
@@ -448,6 +452,7 @@ def main():
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--ratio", default="1")
+    ap.add_argument("--parts", type=int, default=0, help="override the number of partitions (profiling aid)")
     ap.add_argument("--ref-scale", type=float, default=0.01, dest="ref_scale")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -7,6 +7,7 @@
 // send / receive bookkeeping of the exchange.
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <numeric>
@@ -216,16 +217,46 @@ int build(varco_plan *pl, int64_t n, const int64_t *rp0, const int32_t *col0, co
     for (int64_t s = 0; s < pl->H; ++s) pl->brow_slot[fill[where[pl->slot_src[s]]]++] = (int32_t)s;
   }
 
-  // processing orders: longest rows first, so that the tail of a launch is made of short rows
-  auto by_length = [](const std::vector<int64_t> &ptr, int64_t count, std::vector<int32_t> &order) {
-    order.resize(count);
-    std::iota(order.begin(), order.end(), 0);
-    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
-      return (ptr[a + 1] - ptr[a]) > (ptr[b + 1] - ptr[b]);
-    });
+  // processing orders: three classes of rows by number of entries.  Hubs (more than kHubEntries)
+  // get a CTA each.  Short rows (at most kShortEntries) are processed by narrow lane groups, several
+  // rows per warp.  The rest get a full-width group.  Every class list is partition-major (the
+  // kernels sweep partition by partition so that a partition's gathered rows stay in L2) and, inside
+  // a partition, sorted by length, longest first, so that the lanes of a warp run alike.
+  const int64_t kHubEntries = 512, kShortEntries = 8;
+  auto classify = [&](const std::vector<int64_t> &ptr, const std::vector<std::vector<int32_t>> &rows_of_part,
+                      std::vector<int32_t> *lists[3], std::vector<int32_t> *starts[3]) {
+    for (int c = 0; c < 3; ++c) {
+      lists[c]->clear();
+      starts[c]->assign(1, 0);
+    }
+    std::vector<int32_t> tmp[3];
+    for (int q = 0; q < P; ++q) {
+      for (int c = 0; c < 3; ++c) tmp[c].clear();
+      for (int32_t r : rows_of_part[q]) {
+        const int64_t len = ptr[r + 1] - ptr[r];
+        tmp[len > kHubEntries ? 0 : (len <= kShortEntries ? 2 : 1)].push_back(r);
+      }
+      for (int c = 0; c < 3; ++c) {
+        std::stable_sort(tmp[c].begin(), tmp[c].end(),
+                         [&](int32_t a, int32_t b) { return (ptr[a + 1] - ptr[a]) > (ptr[b + 1] - ptr[b]); });
+        lists[c]->insert(lists[c]->end(), tmp[c].begin(), tmp[c].end());
+        starts[c]->push_back((int32_t)lists[c]->size());
+      }
+    }
   };
-  by_length(pl->rp, n, pl->order_f);
-  by_length(pl->rpT, nsrc, pl->order_t);
+  {
+    std::vector<std::vector<int32_t>> rows_of_part(P);
+    for (int q = 0; q < P; ++q)
+      for (int64_t r = pl->part_off[q]; r < pl->part_off[q + 1]; ++r) rows_of_part[q].push_back((int32_t)r);
+    std::vector<int32_t> *lf[3] = {&pl->hub_f, &pl->order_f, &pl->short_f};
+    std::vector<int32_t> *sf[3] = {&pl->hub_f_start, &pl->order_f_start, &pl->short_f_start};
+    classify(pl->rp, rows_of_part, lf, sf);
+    for (int q = 0; q < P; ++q)
+      for (int64_t u = n + slot_base[q]; u < n + slot_base[q + 1]; ++u) rows_of_part[q].push_back((int32_t)u);
+    std::vector<int32_t> *lt[3] = {&pl->hub_t, &pl->order_t, &pl->short_t};
+    std::vector<int32_t> *stt[3] = {&pl->hub_t_start, &pl->order_t_start, &pl->short_t_start};
+    classify(pl->rpT, rows_of_part, lt, stt);
+  }
   return VARCO_OK;
 }
 

@@ -34,7 +34,17 @@ std::vector<ImageItem> image_items(varco_plan *pl) {
           item(pl->brow_ptr, &d.brow_ptr),
           item(pl->brow_slot, &d.brow_slot),
           item(pl->order_f, &d.order_f),
-          item(pl->order_t, &d.order_t)};
+          item(pl->order_t, &d.order_t),
+          item(pl->hub_f, &d.hub_f),
+          item(pl->hub_t, &d.hub_t),
+          item(pl->short_f, &d.short_f),
+          item(pl->short_t, &d.short_t),
+          item(pl->order_f_start, &d.order_f_start),
+          item(pl->order_t_start, &d.order_t_start),
+          item(pl->hub_f_start, &d.hub_f_start),
+          item(pl->hub_t_start, &d.hub_t_start),
+          item(pl->short_f_start, &d.short_f_start),
+          item(pl->short_t_start, &d.short_t_start)};
 }
 
 size_t aligned(size_t b) { return (b + 255) / 256 * 256; }

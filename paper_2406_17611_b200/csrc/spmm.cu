@@ -2,40 +2,84 @@
 //
 // Forward (Algorithm 1, third step; Eq. (2) with one AGGREGATE tap): for every row i of every
 // partition, agg_i = sum_j s_ij u_j where u_j is the exact row of X when the owner of i also
-// owns j and the decompressed halo-slot row otherwise.  Backward: the same kernel walks the
+// owns j and the decompressed halo-slot row otherwise.  Backward: the same kernels walk the
 // transposed structure, sources being dAgg rows and destinations the local rows of dX and the
 // halo-slot gradient rows.
 //
-// One group of G lanes per row (G = 4..32, a whole warp for rows of >= 32 x 16 bytes); every lane
-// owns NCH 16-byte chunks of the feature row, gathers them with 128-bit loads and accumulates in
-// fp32.  Column indices and weights of G entries are loaded cooperatively and broadcast with
-// shuffles; four row gathers are kept in flight per lane.  Rows are taken longest-first.
+// One group of G lanes per row (G = 4..32); every lane owns NCH 16-byte chunks of the feature
+// row, gathers them with 128-bit loads and accumulates in fp32.  Column indices and weights of G
+// entries are loaded cooperatively and broadcast with shuffles; several row gathers are kept in
+// flight per lane.  Rows come in three classes by number of entries: hubs get a CTA each, short
+// rows get narrow lane groups (several rows per warp), the rest a full-width group.
+//
+// Scheduling: the gathers are random 16..512-byte reads bounded by DRAM unless the gathered set
+// stays in L2.  Work is issued partition by partition; the kernels can also split the feature
+// row into panels (task = (partition, panel, row)) so that a partition's gathered set fits in L2,
+// but on the measured workloads the extra passes cost more than the hits return, so the
+// launchers use one panel.
+#include <algorithm>
+
 #include "device_common.cuh"
+#include "kernels.h"
 
 namespace {
 
+struct RowClass {
+  const int32_t *rows;   // row ids, partition-major
+  const int32_t *start;  // [P + 1] first position of every partition in `rows`
+  int count;
+};
+
+struct SpmmArgs {
+  const int64_t *rp;
+  const int32_t *col;
+  const float *val;
+  RowClass hubs, normal, shorts;
+  int P;
+  const void *A0;
+  int64_t lda0;
+  const void *A1;
+  int64_t lda1;
+  int src_split;
+  void *O0;
+  int64_t ldo0;
+  void *O1;
+  int64_t ldo1;
+  int dst_split;
+  int accumulate0;
+  int nv;        // 16-byte chunks per row
+  int panels;    // feature panels
+  int nv_panel;  // chunks per panel
+};
+
+// task id -> (position in the class list, panel); tasks are ordered (partition, panel, row)
+__device__ __forceinline__ void locate(const RowClass &rc, int P, int panels, int64_t task, int &pos, int &panel) {
+  if (panels == 1) {
+    pos = (int)task;
+    panel = 0;
+    return;
+  }
+  int lo = 0, hi = P;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if ((int64_t)__ldg(rc.start + mid) * panels <= task) lo = mid;
+    else hi = mid;
+  }
+  const int s0 = __ldg(rc.start + lo), s1 = __ldg(rc.start + lo + 1);
+  const int64_t local = task - (int64_t)s0 * panels;
+  const int rows_q = s1 - s0;
+  panel = (int)(local / rows_q);
+  pos = s0 + (int)(local % rows_q);
+}
+
+// Accumulate entries [e0, e1) of one row: acc[i][:] += val[e] * chunk (ch_lo + gl + i G) of source col[e].
 template <typename T, int G, int NCH, int UNR>
-__global__ void __launch_bounds__(256)
-    spmm_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col, const float *__restrict__ val,
-                const int32_t *__restrict__ order, int nrows, const T *__restrict__ A0, int64_t lda0,
-                const T *__restrict__ A1, int64_t lda1, int src_split, T *__restrict__ O0, int64_t ldo0,
-                T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv) {
+__device__ __forceinline__ void accumulate_range(int64_t e0, int64_t e1, const int32_t *__restrict__ col,
+                                                 const float *__restrict__ val, const T *__restrict__ A0, int64_t lda0,
+                                                 const T *__restrict__ A1, int64_t lda1, int src_split, int ch_lo,
+                                                 int ch_hi, int gl, unsigned gmask,
+                                                 float (&acc)[NCH][ElemTraits<T>::kVec]) {
   constexpr int V = ElemTraits<T>::kVec;
-  const int tid = blockIdx.x * blockDim.x + threadIdx.x;
-  const int gid = tid / G;
-  const int gl = threadIdx.x % G;
-  if (gid >= nrows) return;
-  const unsigned lane = threadIdx.x % 32;
-  const unsigned gmask = (G == 32) ? 0xFFFFFFFFu : (((1u << G) - 1u) << (lane & ~(unsigned)(G - 1)));
-  const int r = order[gid];
-  const int64_t e0 = rp[r], e1 = rp[r + 1];
-
-  float acc[NCH][V];
-#pragma unroll
-  for (int i = 0; i < NCH; ++i)
-#pragma unroll
-    for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
-
   for (int64_t base = e0; base < e1; base += G) {
     const int cnt = (int)((e1 - base) < (int64_t)G ? (e1 - base) : (int64_t)G);
     int myc = 0;
@@ -58,8 +102,8 @@ __global__ void __launch_bounds__(256)
                                : reinterpret_cast<const uint4 *>(A1 + (int64_t)(c - src_split) * lda1);
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
-          const int ch = gl + i * G;
-          v[u][i] = (live && ch < nv) ? __ldg(src + ch) : make_uint4(0u, 0u, 0u, 0u);
+          const int ch = ch_lo + gl + i * G;
+          v[u][i] = (live && ch < ch_hi) ? __ldg(src + ch) : make_uint4(0u, 0u, 0u, 0u);
         }
         if (!live) w[u] = 0.f;
       }
@@ -74,19 +118,50 @@ __global__ void __launch_bounds__(256)
         }
     }
   }
+}
 
-  uint4 *dst;
-  bool add = false;
+template <typename T>
+__device__ __forceinline__ uint4 *dest_row(int r, T *O0, int64_t ldo0, T *O1, int64_t ldo1, int dst_split,
+                                           int accumulate0, bool &add) {
   if (r < dst_split) {
-    dst = reinterpret_cast<uint4 *>(O0 + (int64_t)r * ldo0);
     add = accumulate0 != 0;
-  } else {
-    dst = reinterpret_cast<uint4 *>(O1 + (int64_t)(r - dst_split) * ldo1);
+    return reinterpret_cast<uint4 *>(O0 + (int64_t)r * ldo0);
   }
+  add = false;
+  return reinterpret_cast<uint4 *>(O1 + (int64_t)(r - dst_split) * ldo1);
+}
+
+template <typename T, int G, int NCH, int UNR>
+__global__ void __launch_bounds__(256)
+    spmm_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col, const float *__restrict__ val,
+                RowClass rc, int P, int panels, int nv_panel, const T *__restrict__ A0, int64_t lda0,
+                const T *__restrict__ A1, int64_t lda1, int src_split, T *__restrict__ O0, int64_t ldo0,
+                T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv) {
+  constexpr int V = ElemTraits<T>::kVec;
+  const int64_t task = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+  const int gl = threadIdx.x % G;
+  if (task >= (int64_t)rc.count * panels) return;
+  const unsigned lane = threadIdx.x % 32;
+  const unsigned gmask = (G == 32) ? 0xFFFFFFFFu : (((1u << G) - 1u) << (lane & ~(unsigned)(G - 1)));
+  int pos, panel;
+  locate(rc, P, panels, task, pos, panel);
+  const int r = __ldg(rc.rows + pos);
+  const int ch_lo = panel * nv_panel;
+  const int ch_hi = min(nv, ch_lo + nv_panel);
+
+  float acc[NCH][V];
+#pragma unroll
+  for (int i = 0; i < NCH; ++i)
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
+  accumulate_range<T, G, NCH, UNR>(rp[r], rp[r + 1], col, val, A0, lda0, A1, lda1, src_split, ch_lo, ch_hi, gl, gmask,
+                                   acc);
+  bool add;
+  uint4 *dst = dest_row<T>(r, O0, ldo0, O1, ldo1, dst_split, accumulate0, add);
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
-    const int ch = gl + i * G;
-    if (ch < nv) {
+    const int ch = ch_lo + gl + i * G;
+    if (ch < ch_hi) {
       if (add) {
         float f[V];
         unpack16(dst[ch], f, T());
@@ -98,49 +173,107 @@ __global__ void __launch_bounds__(256)
   }
 }
 
-struct SpmmArgs {
-  const int64_t *rp;
-  const int32_t *col;
-  const float *val;
-  const int32_t *order;
-  int nrows;
-  const void *A0;
-  int64_t lda0;
-  const void *A1;
-  int64_t lda1;
-  int src_split;
-  void *O0;
-  int64_t ldo0;
-  void *O1;
-  int64_t ldo1;
-  int dst_split;
-  int accumulate0;
-  int nv;
-};
+// Long rows (hubs of a skewed degree distribution): one CTA per (row, panel), every warp takes a
+// contiguous share of the entries, partial sums meet in shared memory and are added in warp order.
+template <typename T, int NCH, int UNR>
+__global__ void __launch_bounds__(256)
+    spmm_hub_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col, const float *__restrict__ val,
+                    RowClass rc, int P, int panels, int nv_panel, const T *__restrict__ A0, int64_t lda0,
+                    const T *__restrict__ A1, int64_t lda1, int src_split, T *__restrict__ O0, int64_t ldo0,
+                    T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv) {
+  extern __shared__ float hub_part[];
+  constexpr int V = ElemTraits<T>::kVec;
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int nwarps = blockDim.x / 32;
+  int pos, panel;
+  locate(rc, P, panels, blockIdx.x, pos, panel);
+  const int r = __ldg(rc.rows + pos);
+  const int ch_lo = panel * nv_panel;
+  const int ch_hi = min(nv, ch_lo + nv_panel);
+  const int64_t e0 = rp[r], e1 = rp[r + 1];
+  const int64_t per = ((e1 - e0 + nwarps - 1) / nwarps + 31) / 32 * 32;
+  const int64_t b0 = e0 + warp * per < e1 ? e0 + warp * per : e1;
+  const int64_t b1 = b0 + per < e1 ? b0 + per : e1;
+  float acc[NCH][V];
+#pragma unroll
+  for (int i = 0; i < NCH; ++i)
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
+  accumulate_range<T, 32, NCH, UNR>(b0, b1, col, val, A0, lda0, A1, lda1, src_split, ch_lo, ch_hi, lane, 0xFFFFFFFFu,
+                                    acc);
+  const int row_floats = nv_panel * V;
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    const int c = lane + i * 32;
+    if (c < nv_panel)
+#pragma unroll
+      for (int j = 0; j < V; ++j) hub_part[(size_t)warp * row_floats + c * V + j] = acc[i][j];
+  }
+  __syncthreads();
+  bool add;
+  uint4 *dst = dest_row<T>(r, O0, ldo0, O1, ldo1, dst_split, accumulate0, add);
+  for (int c = threadIdx.x; c < ch_hi - ch_lo; c += blockDim.x) {
+    float f[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) f[j] = 0.f;
+    if (add) unpack16(dst[ch_lo + c], f, T());
+    for (int w = 0; w < nwarps; ++w)
+#pragma unroll
+      for (int j = 0; j < V; ++j) f[j] += hub_part[(size_t)w * row_floats + c * V + j];
+    dst[ch_lo + c] = pack16(f, T());
+  }
+}
 
-template <typename T, int G, int NCH, int UNR>
-int launch(const SpmmArgs &a, cudaStream_t st) {
-  const int threads = 256;
-  const int64_t total = (int64_t)a.nrows * G;
-  dim3 grid((unsigned)((total + threads - 1) / threads));
-  spmm_kernel<T, G, NCH, UNR><<<grid, threads, 0, st>>>(a.rp, a.col, a.val, a.order, a.nrows, (const T *)a.A0, a.lda0,
-                                                        (const T *)a.A1, a.lda1, a.src_split, (T *)a.O0, a.ldo0,
-                                                        (T *)a.O1, a.ldo1, a.dst_split, a.accumulate0, a.nv);
+template <typename T, int NCH, int UNR>
+int launch_hubs(const SpmmArgs &a, cudaStream_t st) {
+  if (a.hubs.count == 0) return VARCO_OK;
+  constexpr int V = ElemTraits<T>::kVec;
+  const size_t row_bytes = (size_t)a.nv_panel * V * sizeof(float);
+  int warps = 8;
+  while (warps > 1 && warps * row_bytes > 48 * 1024) warps /= 2;
+  spmm_hub_kernel<T, NCH, UNR><<<(unsigned)(a.hubs.count * a.panels), warps * 32, warps * row_bytes, st>>>(
+      a.rp, a.col, a.val, a.hubs, a.P, a.panels, a.nv_panel, (const T *)a.A0, a.lda0, (const T *)a.A1, a.lda1,
+      a.src_split, (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1, a.dst_split, a.accumulate0, a.nv);
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
+template <typename T, int G, int NCH, int UNR>
+int launch_rows(const SpmmArgs &a, const RowClass &rc, cudaStream_t st) {
+  if (rc.count == 0) return VARCO_OK;
+  const int threads = 256;
+  const int64_t total = (int64_t)rc.count * a.panels * G;
+  dim3 grid((unsigned)((total + threads - 1) / threads));
+  spmm_kernel<T, G, NCH, UNR><<<grid, threads, 0, st>>>(a.rp, a.col, a.val, rc, a.P, a.panels, a.nv_panel,
+                                                        (const T *)a.A0, a.lda0, (const T *)a.A1, a.lda1, a.src_split,
+                                                        (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1, a.dst_split,
+                                                        a.accumulate0, a.nv);
+  VARCO_KERNEL_LAUNCHED();
+  return VARCO_OK;
+}
+
+// G/NCH: lanes per row and 16-byte chunks per lane for ordinary rows; GS/NCHS: the same for rows of
+// at most a handful of entries, where narrower groups keep more rows in flight per warp.
+template <typename T, int G, int NCH, int UNR, int GS, int NCHS, int UNRS>
+int launch(const SpmmArgs &a, cudaStream_t st) {
+  if (int rc = launch_hubs<T, NCH, UNR>(a, st)) return rc;
+  if (int rc = launch_rows<T, G, NCH, UNR>(a, a.normal, st)) return rc;
+  return launch_rows<T, GS, NCHS, UNRS>(a, a.shorts, st);
+}
+
 template <typename T>
 int dispatch(const SpmmArgs &a, cudaStream_t st) {
-  const int nv = a.nv;
-  if (nv <= 4) return launch<T, 4, 1, 4>(a, st);
-  if (nv <= 8) return launch<T, 8, 1, 4>(a, st);
-  if (nv <= 16) return launch<T, 16, 1, 4>(a, st);
-  if (nv <= 32) return launch<T, 32, 1, 4>(a, st);
-  if (nv <= 64) return launch<T, 32, 2, 4>(a, st);
-  if (nv <= 96) return launch<T, 32, 3, 4>(a, st);
-  if (nv <= 128) return launch<T, 32, 4, 2>(a, st);
-  if (nv <= 256) return launch<T, 32, 8, 2>(a, st);
+  const int w = a.nv_panel;  // chunks a group has to cover
+  // short-row variants keep one gather per lane in flight: with few entries per row the
+  // parallelism comes from the number of rows resident per SM, i.e. from a low register count
+  if (w <= 4) return launch<T, 4, 1, 4, 4, 1, 2>(a, st);
+  if (w <= 8) return launch<T, 8, 1, 4, 4, 2, 2>(a, st);
+  if (w <= 16) return launch<T, 16, 1, 4, 4, 4, 1>(a, st);
+  if (w <= 32) return launch<T, 32, 1, 4, 8, 4, 1>(a, st);
+  if (w <= 64) return launch<T, 32, 2, 4, 16, 4, 1>(a, st);
+  if (w <= 96) return launch<T, 32, 3, 4, 16, 6, 1>(a, st);
+  if (w <= 128) return launch<T, 32, 4, 2, 32, 4, 1>(a, st);
+  if (w <= 256) return launch<T, 32, 8, 2, 32, 8, 1>(a, st);
   return VARCO_UNSUPPORTED;
 }
 
@@ -150,17 +283,61 @@ int dispatch(const SpmmArgs &a, cudaStream_t st) {
 int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, const void *Xhalo, int64_t ldh, int F,
                           varco_dtype_t dt, void *Agg, int64_t ldagg, cudaStream_t st) {
   const int V = dt == VARCO_F32 ? 4 : 8;
-  SpmmArgs a{pl->d.rp, pl->d.col, pl->d.val, pl->d.order_f, (int)pl->n, X, ldx, Xhalo, ldh, (int)pl->n,
-             Agg,      ldagg,     nullptr,   0,             (int)pl->n, 0, (F + V - 1) / V};
+  const int nv = (F + V - 1) / V;
+  SpmmArgs a{};
+  a.rp = pl->d.rp;
+  a.col = pl->d.col;
+  a.val = pl->d.val;
+  a.hubs = RowClass{pl->d.hub_f, pl->d.hub_f_start, (int)pl->hub_f.size()};
+  a.normal = RowClass{pl->d.order_f, pl->d.order_f_start, (int)pl->order_f.size()};
+  a.shorts = RowClass{pl->d.short_f, pl->d.short_f_start, (int)pl->short_f.size()};
+  a.P = pl->P;
+  a.A0 = X;
+  a.lda0 = ldx;
+  a.A1 = Xhalo;
+  a.lda1 = ldh;
+  a.src_split = (int)pl->n;
+  a.O0 = Agg;
+  a.ldo0 = ldagg;
+  a.O1 = nullptr;
+  a.ldo1 = 0;
+  a.dst_split = (int)pl->n;
+  a.accumulate0 = 0;
+  a.nv = nv;
+  a.panels = 1;
+  a.nv_panel = nv;
   return dt == VARCO_F32 ? dispatch<float>(a, st) : dispatch<__nv_bfloat16>(a, st);
 }
 
 // Transposed aggregation: for a source u, g_u = sum over the rows i that use it of s_iu dAgg[i];
 // u < n lands in dX[u] (added to what is there when `accumulate`), u >= n in Ghalo[u - n].
+// Every source of partition q is used by rows of q only, so the gathered set of a partition is
+// its own block of dAgg: panels are chosen so that this block stays in L2.
 int varco_launch_spmm_bwd(const varco_plan *pl, const void *dAgg, int64_t ldd, int F, varco_dtype_t dt, void *dX,
                           int64_t ldx, int accumulate, void *Ghalo, int64_t ldh, cudaStream_t st) {
   const int V = dt == VARCO_F32 ? 4 : 8;
-  SpmmArgs a{pl->d.rpT, pl->d.colT, pl->d.valT, pl->d.order_t, (int)(pl->n + pl->H), dAgg, ldd, dAgg, ldd,
-             (int)pl->n, dX, ldx, Ghalo, ldh, (int)pl->n, accumulate, (F + V - 1) / V};
+  const int nv = (F + V - 1) / V;
+  SpmmArgs a{};
+  a.rp = pl->d.rpT;
+  a.col = pl->d.colT;
+  a.val = pl->d.valT;
+  a.hubs = RowClass{pl->d.hub_t, pl->d.hub_t_start, (int)pl->hub_t.size()};
+  a.normal = RowClass{pl->d.order_t, pl->d.order_t_start, (int)pl->order_t.size()};
+  a.shorts = RowClass{pl->d.short_t, pl->d.short_t_start, (int)pl->short_t.size()};
+  a.P = pl->P;
+  a.A0 = dAgg;
+  a.lda0 = ldd;
+  a.A1 = dAgg;
+  a.lda1 = ldd;
+  a.src_split = (int)pl->n;
+  a.O0 = dX;
+  a.ldo0 = ldx;
+  a.O1 = Ghalo;
+  a.ldo1 = ldh;
+  a.dst_split = (int)pl->n;
+  a.accumulate0 = accumulate;
+  a.nv = nv;
+  a.panels = 1;
+  a.nv_panel = nv;
   return dt == VARCO_F32 ? dispatch<float>(a, st) : dispatch<__nv_bfloat16>(a, st);
 }

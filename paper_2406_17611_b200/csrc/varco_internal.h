@@ -28,9 +28,17 @@ struct varco_dev_image {
   const int32_t *brow = nullptr;
   const int32_t *brow_ptr = nullptr;
   const int32_t *brow_slot = nullptr;
-  // rows sorted by descending number of entries (forward rows; transposed sources)
+  // processing orders (forward rows; transposed sources): ordinary rows partition by partition,
+  // and the long rows that get a CTA each
   const int32_t *order_f = nullptr;
   const int32_t *order_t = nullptr;
+  const int32_t *hub_f = nullptr;
+  const int32_t *hub_t = nullptr;
+  const int32_t *short_f = nullptr;
+  const int32_t *short_t = nullptr;
+  // [P + 1] first position of every partition in the class lists above
+  const int32_t *order_f_start = nullptr, *order_t_start = nullptr, *hub_f_start = nullptr, *hub_t_start = nullptr,
+                *short_f_start = nullptr, *short_t_start = nullptr;
 };
 
 struct varco_profile;  // CUDA-event bookkeeping, defined in runtime.cu
@@ -42,7 +50,8 @@ struct varco_plan {
   std::vector<int64_t> new_to_old, part_off, counts, send_base, halo_ids;
   // host copies of the device image
   std::vector<int32_t> row_gid, col, colT, slot_gid, slot_src, slot_sendpos, brow, brow_ptr, brow_slot;
-  std::vector<int32_t> order_f, order_t;
+  std::vector<int32_t> order_f, order_t, hub_f, hub_t, short_f, short_t;
+  std::vector<int32_t> order_f_start, order_t_start, hub_f_start, hub_t_start, short_f_start, short_t_start;
   std::vector<int64_t> rp, rpT;
   std::vector<float> val, valT;
   // device image

@@ -180,6 +180,45 @@ def test_degenerate_graphs(orc):
             plan.close()
 
 
+@pytest.mark.parametrize("bf16,F_in,F_out", [(False, 64, 32), (True, 256, 64), (True, 100, 47)])
+def test_hub_rows(orc, bf16, F_in, F_out):
+    """Rows and sources with thousands of entries take the CTA-per-row path of the aggregation."""
+    n, P = 6000, 4
+    rng = np.random.default_rng(3)
+    hubs = np.repeat(np.arange(3, dtype=np.int64), n - 3)
+    others = np.tile(np.arange(3, n, dtype=np.int64), 3)
+    ring = np.arange(n, dtype=np.int64)
+    rp, col = synth._csr_from_pairs(n, np.concatenate([hubs, ring]), np.concatenate([others, (ring + 1) % n]))
+    part = synth.partition_random_equal(n, P, 5)
+    dt = torch.bfloat16 if bf16 else torch.float32
+    X = synth.normal_features(n, F_in, 1, bf16)
+    Wn = synth.glorot_uniform(F_in, F_out, 2, bf16)
+    Ws = synth.glorot_uniform(F_in, F_out, 3, bf16)
+    b = (0.1 * rng.standard_normal(F_out)).astype(np.float32)
+    dY = rng.standard_normal((n, F_out)).astype(np.float32)
+    dY = synth.bf16_round(dY) if bf16 else dY
+    plan = vb.Plan(rp, col, part, P, "sage").upload()
+    g = orc.graph(rp, col, part, P, "sage")
+    perm = plan.perm()
+    ws = plan.workspace(F_in, F_out, vb.BF16 if bf16 else vb.F32)
+    Xd = to_device_rows(X, perm, dt)
+    for ratio in [(1, 1), (4, 1)]:
+        key = (9, 1, 0)
+        Y, Agg, _ = vb.varco_layer_fwd(plan, Xd, dev_weights(Ws, dt), dev_weights(Wn, dt),
+                                       dev_weights(b, torch.float32), True, ratio, key, ws, F_in=F_in)
+        Yr, Aggr, _ = g.layer_fwd(X, Ws, Wn, b, True, ratio, key)
+        assert rel_err(to_host_rows(Agg, perm, F_in), Aggr) <= TOL[dt]
+        assert rel_err(to_host_rows(Y, perm, F_out), Yr) <= TOL[dt]
+        Yd = to_device_rows(Yr.astype(np.float32), perm, dt)
+        dX, dWs, dWn, db, _ = vb.varco_layer_bwd(plan, Xd, Yd, Agg, dev_weights(Ws, dt), dev_weights(Wn, dt),
+                                                 to_device_rows(dY, perm, dt), True, ratio, key, ws, F_in=F_in)
+        rX, rWs, rWn, rb, _ = g.layer_bwd(X, to_host_rows(Yd, perm, F_out), Ws, Wn, dY, True, ratio, key)
+        assert vb.varco_workspace_status(ws) == 0
+        assert rel_err(to_host_rows(dX, perm, F_in), rX) <= TOL[dt]
+        assert rel_err(host64(dWn), rWn) <= TOL[dt] and rel_err(host64(dWs), rWs) <= TOL[dt]
+    plan.close()
+
+
 def test_backward_is_reproducible(cases):
     """The ordered (atomic-free) gradient accumulation gives bit-identical results run to run."""
     case = cases("c2r", 0.05)
