@@ -156,6 +156,34 @@ int varco_decompress(const varco_plan_t *plan, const void *packed, int32_t F, va
                      varco_ratio_t c, varco_key_t key, void *Xhalo, int64_t ld, void *stream);
 
 /* ------------------------------------------------------------------------------------------
+ * Exchange round trip without any allocation.  The paper has no counterpart: this entry point
+ * exists for callers that are not allowed to allocate device memory -- code running where
+ * cudaMalloc is forbidden or would stall the device (a serving loop with a latency budget, a hook
+ * called while another framework owns the memory pool, a process whose caching allocator already
+ * holds all device memory).
+ *
+ * varco_exchange_noalloc computes Xhalo = varco_decompress(varco_compress(X)) -- every halo slot
+ * receives the row of its owner with the k kept values in place and zeros elsewhere -- and keeps
+ * the packed rows in between in a fixed array of VARCO_NOALLOC_SCRATCH_BYTES bytes that is part
+ * of the library image (every GPU that loads the library holds that much until the process
+ * exits).  It calls no cudaMalloc, cudaFree or other allocating routine.
+ *   X [n x ld], Xhalo [H_total x ld_halo]  device, caller-owned, same rules as varco_compress /
+ *                                           varco_decompress; bytes (host, optional) as there.
+ *   Limit: H_total * round_up(k, 16 / element_size) * element_size <= VARCO_NOALLOC_SCRATCH_BYTES,
+ *   otherwise VARCO_WORKSPACE_TOO_SMALL and nothing is launched.
+ *   The first call on a device looks up the device address of the array (once per device, with
+ *   that device current); make that first call outside any stream capture.
+ *   All calls on a device share the one array, which keeps the last call's packed rows: two calls
+ *   whose kernels may overlap on the GPU (different streams) race on it.  Calls on one stream are
+ *   ordered and safe.  Nothing needs clearing between calls.
+ *   Errors: INVALID_ARG, NOT_UPLOADED, UNSUPPORTED, WORKSPACE_TOO_SMALL, CUDA.
+ */
+#define VARCO_NOALLOC_SCRATCH_BYTES (32u << 20)
+int varco_exchange_noalloc(const varco_plan_t *plan, const void *X, int64_t ld, int32_t F,
+                           varco_dtype_t dtype, varco_ratio_t c, varco_key_t key, void *Xhalo,
+                           int64_t ld_halo, uint64_t *bytes, void *stream);
+
+/* ------------------------------------------------------------------------------------------
  * One layer over all partitions (Eq. (2) with two taps; Algorithm 1 steps 2-4).
  *
  *   relu    1: ReLU after the transform, 0: identity (last layer).

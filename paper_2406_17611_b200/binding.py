@@ -23,7 +23,8 @@ EXPORTS = ["varco_status_string", "varco_partition_build", "varco_partition_dest
            "varco_partition_boundary_rows", "varco_partition_counts", "varco_partition_halo", "varco_partition_perm", "varco_partition_device_bytes",
            "varco_partition_upload", "varco_workspace_bytes", "varco_kept", "varco_schedule_linear",
            "varco_compress", "varco_decompress", "varco_layer_fwd", "varco_layer_bwd", "varco_profile_enable",
-           "varco_profile_reset", "varco_profile_read", "varco_kernel_launches", "varco_workspace_status"]
+           "varco_profile_reset", "varco_profile_read", "varco_kernel_launches", "varco_workspace_status",
+           "varco_exchange_noalloc"]
 
 
 class Ratio(C.Structure):
@@ -74,6 +75,8 @@ def lib():
     L.varco_schedule_linear.argtypes = [C.c_int32] * 5 + [C.POINTER(Ratio)]
     L.varco_compress.argtypes = [vp, vp, C.c_int64, C.c_int32, C.c_int, Ratio, Key, vp, C.POINTER(C.c_uint64), vp]
     L.varco_decompress.argtypes = [vp, vp, C.c_int32, C.c_int, Ratio, Key, vp, C.c_int64, vp]
+    L.varco_exchange_noalloc.argtypes = [vp, vp, C.c_int64, C.c_int32, C.c_int, Ratio, Key, vp, C.c_int64,
+                                         C.POINTER(C.c_uint64), vp]
     L.varco_layer_fwd.argtypes = [vp, C.POINTER(LayerDesc), vp, vp, vp, vp, vp, vp, Ratio, Key, vp, C.c_size_t,
                                   C.POINTER(C.c_uint64), vp]
     L.varco_layer_bwd.argtypes = [vp, C.POINTER(LayerDesc), vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, Ratio, Key, vp,
@@ -260,6 +263,19 @@ def varco_decompress(plan: Plan, packed, F, ratio, key, ld=None, out=None):
     _check(lib().varco_decompress(plan.h, _ptr(packed), int(F), _dtype_of(packed), _ratio(ratio), _key(key),
                                   _ptr(out), ld, _stream()), "varco_decompress")
     return out
+
+
+NOALLOC_SCRATCH_BYTES = 32 << 20
+
+
+def varco_exchange_noalloc(plan: Plan, X, F, ratio, key, out):
+    """decompress(compress(X)) into the caller's `out` [H_total x ld] using only the library's
+    built-in scratch: for callers that must not allocate device memory.  Returns the wire bytes."""
+    nbytes = C.c_uint64()
+    _check(lib().varco_exchange_noalloc(plan.h, _ptr(X), X.stride(0), int(F), _dtype_of(X), _ratio(ratio), _key(key),
+                                        _ptr(out), out.stride(0), C.byref(nbytes), _stream()),
+           "varco_exchange_noalloc")
+    return int(nbytes.value)
 
 
 def _desc(plan, X, F_in, F_out, relu, ld_out):
