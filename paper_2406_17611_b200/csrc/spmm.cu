@@ -72,40 +72,40 @@ __device__ __forceinline__ void locate(const RowClass &rc, int P, int panels, in
   pos = s0 + (int)(local % rows_q);
 }
 
-// Accumulate entries [e0, e1) of one row: acc[i][:] += val[e] * chunk (ch_lo + gl + i G) of source col[e].
-template <typename T, int G, int NCH, int UNR>
-__device__ __forceinline__ void accumulate_range(int64_t e0, int64_t e1, const int32_t *__restrict__ col,
-                                                 const float *__restrict__ val, const T *__restrict__ A0, int64_t lda0,
-                                                 const T *__restrict__ A1, int64_t lda1, int src_split, int ch_lo,
-                                                 int ch_hi, int gl, unsigned gmask,
-                                                 float (&acc)[NCH][ElemTraits<T>::kVec]) {
+// Where the gathers read from: sources below `split` are rows of A0, the others rows of A1.  The A1 base is
+// stored pre-offset by -split rows, so that both cases are base + c * stride.
+struct GatherSrc {
+  const uint4 *b0, *b1s;   // in 16-byte units
+  int ld0, ld1;            // row strides in 16-byte units
+  int split;
+};
+
+// Accumulate `len` entries of one row: acc[i][:] += val[e] * chunk (ch_lo + gl + i G) of source col[e].
+// FULL: the group covers exactly the row's chunks, no bounds test on the chunk index.
+// Entries are taken G at a time; lanes beyond the last entry of a batch hold a valid column with weight
+// zero, so that the inner loop needs no per-entry predicate.
+template <typename T, int G, int NCH, int UNR, bool FULL>
+__device__ __forceinline__ void accumulate_range(const int32_t *__restrict__ colp, const float *__restrict__ valp,
+                                                 int len, const GatherSrc &gs, int ch_lo, int ch_hi, int gl,
+                                                 unsigned gmask, float (&acc)[NCH][ElemTraits<T>::kVec]) {
   constexpr int V = ElemTraits<T>::kVec;
-  for (int64_t base = e0; base < e1; base += G) {
-    const int cnt = (int)((e1 - base) < (int64_t)G ? (e1 - base) : (int64_t)G);
-    int myc = 0;
-    float myw = 0.f;
-    if (gl < cnt) {
-      myc = __ldg(col + base + gl);
-      myw = __ldg(val + base + gl);
-    }
+  for (int base = 0; base < len; base += G) {
+    const int cnt = min(G, len - base);
+    const int mine = base + min(gl, cnt - 1);
+    const int myc = __ldg(colp + mine);
+    const float myw = gl < cnt ? __ldg(valp + mine) : 0.f;
     for (int t = 0; t < cnt; t += UNR) {
       uint4 v[UNR][NCH];
       float w[UNR];
 #pragma unroll
       for (int u = 0; u < UNR; ++u) {
-        const int tt = t + u;
-        const int c = __shfl_sync(gmask, myc, tt, G);
-        w[u] = __shfl_sync(gmask, myw, tt, G);
-        const bool live = tt < cnt;
-        const uint4 *src = (c < src_split)
-                               ? reinterpret_cast<const uint4 *>(A0 + (int64_t)c * lda0)
-                               : reinterpret_cast<const uint4 *>(A1 + (int64_t)(c - src_split) * lda1);
+        const int c = __shfl_sync(gmask, myc, t + u, G);
+        w[u] = __shfl_sync(gmask, myw, t + u, G);
+        const bool loc = c < gs.split;
+        const uint4 *src = (loc ? gs.b0 : gs.b1s) + (int64_t)c * (loc ? gs.ld0 : gs.ld1) + (ch_lo + gl);
 #pragma unroll
-        for (int i = 0; i < NCH; ++i) {
-          const int ch = ch_lo + gl + i * G;
-          v[u][i] = (live && ch < ch_hi) ? __ldg(src + ch) : make_uint4(0u, 0u, 0u, 0u);
-        }
-        if (!live) w[u] = 0.f;
+        for (int i = 0; i < NCH; ++i)
+          v[u][i] = (FULL || ch_lo + gl + i * G < ch_hi) ? __ldg(src + i * G) : make_uint4(0u, 0u, 0u, 0u);
       }
 #pragma unroll
       for (int u = 0; u < UNR; ++u)
@@ -131,11 +131,10 @@ __device__ __forceinline__ uint4 *dest_row(int r, T *O0, int64_t ldo0, T *O1, in
   return reinterpret_cast<uint4 *>(O1 + (int64_t)(r - dst_split) * ldo1);
 }
 
-template <typename T, int G, int NCH, int UNR>
+template <typename T, int G, int NCH, int UNR, bool FULL>
 __global__ void __launch_bounds__(256)
     spmm_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col, const float *__restrict__ val,
-                RowClass rc, int P, int panels, int nv_panel, const T *__restrict__ A0, int64_t lda0,
-                const T *__restrict__ A1, int64_t lda1, int src_split, T *__restrict__ O0, int64_t ldo0,
+                RowClass rc, int P, int panels, int nv_panel, GatherSrc gs, T *__restrict__ O0, int64_t ldo0,
                 T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv) {
   constexpr int V = ElemTraits<T>::kVec;
   const int64_t task = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
@@ -154,8 +153,8 @@ __global__ void __launch_bounds__(256)
   for (int i = 0; i < NCH; ++i)
 #pragma unroll
     for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
-  accumulate_range<T, G, NCH, UNR>(rp[r], rp[r + 1], col, val, A0, lda0, A1, lda1, src_split, ch_lo, ch_hi, gl, gmask,
-                                   acc);
+  const int64_t e0 = rp[r];
+  accumulate_range<T, G, NCH, UNR, FULL>(col + e0, val + e0, (int)(rp[r + 1] - e0), gs, ch_lo, ch_hi, gl, gmask, acc);
   bool add;
   uint4 *dst = dest_row<T>(r, O0, ldo0, O1, ldo1, dst_split, accumulate0, add);
 #pragma unroll
@@ -175,11 +174,10 @@ __global__ void __launch_bounds__(256)
 
 // Long rows (hubs of a skewed degree distribution): one CTA per (row, panel), every warp takes a
 // contiguous share of the entries, partial sums meet in shared memory and are added in warp order.
-template <typename T, int NCH, int UNR>
+template <typename T, int NCH, int UNR, bool FULL>
 __global__ void __launch_bounds__(256)
     spmm_hub_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col, const float *__restrict__ val,
-                    RowClass rc, int P, int panels, int nv_panel, const T *__restrict__ A0, int64_t lda0,
-                    const T *__restrict__ A1, int64_t lda1, int src_split, T *__restrict__ O0, int64_t ldo0,
+                    RowClass rc, int P, int panels, int nv_panel, GatherSrc gs, T *__restrict__ O0, int64_t ldo0,
                     T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv) {
   extern __shared__ float hub_part[];
   constexpr int V = ElemTraits<T>::kVec;
@@ -199,8 +197,9 @@ __global__ void __launch_bounds__(256)
   for (int i = 0; i < NCH; ++i)
 #pragma unroll
     for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
-  accumulate_range<T, 32, NCH, UNR>(b0, b1, col, val, A0, lda0, A1, lda1, src_split, ch_lo, ch_hi, lane, 0xFFFFFFFFu,
-                                    acc);
+  if (b1 > b0)
+    accumulate_range<T, 32, NCH, UNR, FULL>(col + b0, val + b0, (int)(b1 - b0), gs, ch_lo, ch_hi, lane, 0xFFFFFFFFu,
+                                            acc);
   const int row_floats = nv_panel * V;
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
@@ -224,6 +223,18 @@ __global__ void __launch_bounds__(256)
   }
 }
 
+template <typename T>
+GatherSrc gather_src(const SpmmArgs &a) {
+  constexpr int V = ElemTraits<T>::kVec;
+  GatherSrc gs;
+  gs.b0 = reinterpret_cast<const uint4 *>(a.A0);
+  gs.ld0 = (int)(a.lda0 / V);
+  gs.ld1 = (int)(a.lda1 / V);
+  gs.b1s = reinterpret_cast<const uint4 *>(a.A1) - (int64_t)a.src_split * gs.ld1;
+  gs.split = a.src_split;
+  return gs;
+}
+
 template <typename T, int NCH, int UNR>
 int launch_hubs(const SpmmArgs &a, cudaStream_t st) {
   if (a.hubs.count == 0) return VARCO_OK;
@@ -231,9 +242,15 @@ int launch_hubs(const SpmmArgs &a, cudaStream_t st) {
   const size_t row_bytes = (size_t)a.nv_panel * V * sizeof(float);
   int warps = 8;
   while (warps > 1 && warps * row_bytes > 48 * 1024) warps /= 2;
-  spmm_hub_kernel<T, NCH, UNR><<<(unsigned)(a.hubs.count * a.panels), warps * 32, warps * row_bytes, st>>>(
-      a.rp, a.col, a.val, a.hubs, a.P, a.panels, a.nv_panel, (const T *)a.A0, a.lda0, (const T *)a.A1, a.lda1,
-      a.src_split, (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1, a.dst_split, a.accumulate0, a.nv);
+  const dim3 grid((unsigned)(a.hubs.count * a.panels));
+  if (a.panels == 1 && a.nv == 32 * NCH)
+    spmm_hub_kernel<T, NCH, UNR, true><<<grid, warps * 32, warps * row_bytes, st>>>(
+        a.rp, a.col, a.val, a.hubs, a.P, a.panels, a.nv_panel, gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1,
+        a.dst_split, a.accumulate0, a.nv);
+  else
+    spmm_hub_kernel<T, NCH, UNR, false><<<grid, warps * 32, warps * row_bytes, st>>>(
+        a.rp, a.col, a.val, a.hubs, a.P, a.panels, a.nv_panel, gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1,
+        a.dst_split, a.accumulate0, a.nv);
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
@@ -244,10 +261,14 @@ int launch_rows(const SpmmArgs &a, const RowClass &rc, cudaStream_t st) {
   const int threads = 256;
   const int64_t total = (int64_t)rc.count * a.panels * G;
   dim3 grid((unsigned)((total + threads - 1) / threads));
-  spmm_kernel<T, G, NCH, UNR><<<grid, threads, 0, st>>>(a.rp, a.col, a.val, rc, a.P, a.panels, a.nv_panel,
-                                                        (const T *)a.A0, a.lda0, (const T *)a.A1, a.lda1, a.src_split,
-                                                        (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1, a.dst_split,
-                                                        a.accumulate0, a.nv);
+  if (a.panels == 1 && a.nv == G * NCH)
+    spmm_kernel<T, G, NCH, UNR, true><<<grid, threads, 0, st>>>(a.rp, a.col, a.val, rc, a.P, a.panels, a.nv_panel,
+                                                                gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1,
+                                                                a.dst_split, a.accumulate0, a.nv);
+  else
+    spmm_kernel<T, G, NCH, UNR, false><<<grid, threads, 0, st>>>(a.rp, a.col, a.val, rc, a.P, a.panels, a.nv_panel,
+                                                                 gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1,
+                                                                 a.ldo1, a.dst_split, a.accumulate0, a.nv);
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
