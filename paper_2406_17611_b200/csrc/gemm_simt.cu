@@ -122,16 +122,37 @@ __global__ void reduce_partials_kernel(const float *__restrict__ partial, int64_
   out[i] = s;
 }
 
-// partial[z][c] = sum over the rows of chunk z of dZ[row][c]
+// partial[z][c] = sum over the rows of chunk z of dZ[row][c].  Block = 32 x 8 threads: x owns a 16-byte
+// chunk of columns, y strides over the rows; the eight row-partials meet in shared memory in y order.
 template <typename T>
-__global__ void colsum_kernel(const T *__restrict__ dZ, int64_t ld, int rows, int N, int row_chunk,
-                              float *__restrict__ partial) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= N) return;
+__global__ void __launch_bounds__(256) colsum_kernel(const T *__restrict__ dZ, int64_t ld, int rows, int N, int nv,
+                                                     int row_chunk, float *__restrict__ partial) {
+  constexpr int V = ElemTraits<T>::kVec;
+  __shared__ float red[8][32][V + 1];
+  const int ch = blockIdx.x * 32 + threadIdx.x;
   const int r0 = blockIdx.y * row_chunk, r1 = min(rows, r0 + row_chunk);
-  float s = 0.f;
-  for (int r = r0; r < r1; ++r) s += ldf(dZ + (int64_t)r * ld + c);
-  partial[(int64_t)blockIdx.y * N + c] = s;
+  float s[V];
+#pragma unroll
+  for (int j = 0; j < V; ++j) s[j] = 0.f;
+  if (ch < nv)
+    for (int r = r0 + threadIdx.y; r < r1; r += 8) {
+      float f[V];
+      unpack16(__ldg(reinterpret_cast<const uint4 *>(dZ + (int64_t)r * ld) + ch), f, T());
+#pragma unroll
+      for (int j = 0; j < V; ++j) s[j] += f[j];
+    }
+#pragma unroll
+  for (int j = 0; j < V; ++j) red[threadIdx.y][threadIdx.x][j] = s[j];
+  __syncthreads();
+  if (threadIdx.y == 0 && ch < nv) {
+#pragma unroll
+    for (int j = 0; j < V; ++j) {
+      float t = 0.f;
+      for (int y = 0; y < 8; ++y) t += red[y][threadIdx.x][j];
+      const int c = ch * V + j;
+      if (c < N) partial[(int64_t)blockIdx.y * N + c] = t;
+    }
+  }
 }
 
 // dZ = dY where Y > 0, else 0; 16 bytes per thread
@@ -234,11 +255,14 @@ int varco_colsum(int n, int F_out, varco_dtype_t dt, const void *dZ, int64_t ldd
   int chunk = (n + splits - 1) / splits;
   if (chunk < 1) chunk = 1;
   splits = (n + chunk - 1) / chunk;
-  dim3 grid((F_out + 127) / 128, splits);
+  const int V = dt == VARCO_F32 ? 4 : 8;
+  const int nv = (F_out + V - 1) / V;
+  dim3 grid((nv + 31) / 32, splits), block(32, 8);
   if (dt == VARCO_F32)
-    colsum_kernel<float><<<grid, 128, 0, st>>>((const float *)dZ, lddz, n, F_out, chunk, scratch);
+    colsum_kernel<float><<<grid, block, 0, st>>>((const float *)dZ, lddz, n, F_out, nv, chunk, scratch);
   else
-    colsum_kernel<__nv_bfloat16><<<grid, 128, 0, st>>>((const __nv_bfloat16 *)dZ, lddz, n, F_out, chunk, scratch);
+    colsum_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16 *)dZ, lddz, n, F_out, nv, chunk,
+                                                         scratch);
   VARCO_KERNEL_LAUNCHED();
   reduce_partials_kernel<<<(F_out + 255) / 256, 256, 0, st>>>(scratch, F_out, splits, out);
   VARCO_KERNEL_LAUNCHED();
