@@ -104,6 +104,11 @@ template <> struct ElemTraits<__nv_bfloat16> {
   __device__ static __forceinline__ __nv_bfloat16 from_f(float v) { return __float2bfloat16_rn(v); }
 };
 
+// raw element type of the same width, for bit-exact copies
+template <typename T> struct ElemBits;
+template <> struct ElemBits<float> { typedef uint32_t type; };
+template <> struct ElemBits<__nv_bfloat16> { typedef uint16_t type; };
+
 // unpack 16 bytes of T into floats
 __device__ __forceinline__ void unpack16(const uint4 &v, float (&f)[4], float) {
   f[0] = __uint_as_float(v.x);
@@ -132,6 +137,29 @@ __device__ __forceinline__ uint4 pack16(const float (&f)[8], __nv_bfloat16) {
   return make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]),
                     pack_bf16x2(f[6], f[7]));
 }
+
+#ifdef __CUDACC__
+// lanes of the G-lane group this thread belongs to (G a power of two, groups aligned inside the warp)
+template <int G> __device__ __forceinline__ unsigned group_mask() {
+  if (G == 32) return 0xFFFFFFFFu;
+  const unsigned lane = threadIdx.x & 31u;
+  return ((1u << G) - 1u) << (lane & ~(unsigned)(G - 1));
+}
+
+// Round keys of one row, computed by six lanes of the group and shared by shuffle (G >= 8).
+template <int G>
+__device__ __forceinline__ void init_perm(vperm::RowPerm &pm, uint64_t lkey, uint32_t node, uint32_t F, int h, int gl,
+                                          unsigned gmask) {
+  const uint64_t a = vperm::mix(lkey + (uint64_t)node);
+  uint32_t mine = 0;
+  if (gl < 6) mine = (uint32_t)(vperm::mix(a + (uint64_t)(gl + 1) * vperm::kPhi64) >> 32) * vperm::kGold32;
+#pragma unroll
+  for (int i = 0; i < 6; ++i) pm.rkg[i] = __shfl_sync(gmask, mine, i, G);
+  pm.F = F;
+  pm.h = h;
+}
+
+#endif
 
 static inline int64_t round_up64(int64_t a, int64_t b) { return (a + b - 1) / b * b; }
 

@@ -24,25 +24,6 @@ namespace {
 
 template <typename E> struct VecOf { static constexpr int kVec = 16 / (int)sizeof(E); };
 
-template <int G> __device__ __forceinline__ unsigned group_mask() {
-  if (G == 32) return 0xFFFFFFFFu;
-  const unsigned lane = threadIdx.x & 31u;
-  return ((1u << G) - 1u) << (lane & ~(unsigned)(G - 1));
-}
-
-// Round keys of one row, computed by six lanes of the group and shared by shuffle.
-template <int G>
-__device__ __forceinline__ void init_perm(vperm::RowPerm &pm, uint64_t lkey, uint32_t node, uint32_t F, int h, int gl,
-                                          unsigned gmask) {
-  const uint64_t a = vperm::mix(lkey + (uint64_t)node);
-  uint32_t mine = 0;
-  if (gl < 6) mine = (uint32_t)(vperm::mix(a + (uint64_t)(gl + 1) * vperm::kPhi64) >> 32) * vperm::kGold32;
-#pragma unroll
-  for (int i = 0; i < 6; ++i) pm.rkg[i] = __shfl_sync(gmask, mine, i, G);
-  pm.F = F;
-  pm.h = h;
-}
-
 __device__ __forceinline__ uint32_t wire_pos(const vperm::RowPerm &pm, int m, bool identity) {
   return identity ? (uint32_t)m : pm.pi((uint32_t)m);
 }
@@ -169,38 +150,29 @@ __global__ void __launch_bounds__(256) decompress_slots_kernel(const E *__restri
 }
 
 // ------------------------------------------------------------------------------------------
-// Backward, receiver side (now the sender of gradients), k < F.  One group per halo slot: the
-// slot's gradient row is compressed with the forward's permutation; packed rows in slot order.
+// Receiver side, sparse form.  Instead of a dense row with F - k zeros, the slot keeps its k
+// received values next to the positions they belong to: pair m = (value m, pi(m)).  The
+// aggregation then reads k pairs per remote neighbour instead of F elements.  bf16: one 32-bit
+// word per pair (value in the low half, position in the high half); fp32: two words.
 template <typename E, int G>
-__global__ void __launch_bounds__(256) compress_slots_kernel(const E *__restrict__ Gh, int64_t ld, int F, int k, int h,
-                                                             uint64_t lkey, const int32_t *__restrict__ slot_gid,
-                                                             int H, E *__restrict__ packed, int64_t kstride) {
-  extern __shared__ uint4 smem_u4[];
-  constexpr int V = VecOf<E>::kVec;
-  const int nv = (F + V - 1) / V;
-  const int kv = (k + V - 1) / V;
-  const int grp = threadIdx.x / G, gl = threadIdx.x % G;
-  const int slot = blockIdx.x * (blockDim.x / G) + grp;
+__global__ void __launch_bounds__(256) expand_slots_kernel(const E *__restrict__ packed, int64_t kstride, int F, int k,
+                                                           int h, uint64_t lkey, const int32_t *__restrict__ slot_gid,
+                                                           int H, uint32_t *__restrict__ pairs, int64_t pstride) {
+  const int slot = (blockIdx.x * blockDim.x + threadIdx.x) / G;
+  const int gl = threadIdx.x % G;
   if (slot >= H) return;
   const unsigned gmask = group_mask<G>();
-  uint4 *srow4 = smem_u4 + (size_t)grp * (nv + kv);
-  uint4 *zrow4 = srow4 + nv;
-  const E *srow = reinterpret_cast<const E *>(srow4);
-  E *zrow = reinterpret_cast<E *>(zrow4);
-  const uint4 *src = reinterpret_cast<const uint4 *>(Gh + (int64_t)slot * ld);
-  for (int v = gl; v < nv; v += G) srow4[v] = __ldg(src + v);
   vperm::RowPerm pm;
   init_perm<G>(pm, lkey, (uint32_t)slot_gid[slot], (uint32_t)F, h, gl, gmask);
-  const bool identity = k == F;
-  __syncwarp(gmask);
-  for (int m = gl; m < kv * V; m += G) zrow[m] = m < k ? srow[wire_pos(pm, m, identity)] : (E)0;
-  __syncwarp(gmask);
-  E *dst = packed + (int64_t)slot * kstride;
-  if (((kstride * (int64_t)sizeof(E)) & 15) == 0) {
-    uint4 *dst4 = reinterpret_cast<uint4 *>(dst);
-    for (int v = gl; v < kv; v += G) dst4[v] = zrow4[v];
-  } else {
-    for (int m = gl; m < k; m += G) dst[m] = zrow[m];
+  const E *z = packed + (int64_t)slot * kstride;
+  for (int m = gl; m < pstride; m += G) {
+    const uint32_t pos = m < k ? pm.pi((uint32_t)m) : 0u;
+    const uint32_t v = m < k ? (uint32_t)z[m] : 0u;   // padding pairs: value 0 at position 0
+    if (sizeof(E) == 2) {
+      pairs[(int64_t)slot * pstride + m] = v | (pos << 16);
+    } else {
+      reinterpret_cast<uint2 *>(pairs)[(int64_t)slot * pstride + m] = make_uint2(v, pos);
+    }
   }
 }
 
@@ -381,22 +353,25 @@ int varco_launch_decompress_slots(const varco_plan *pl, const void *packed, int6
   return VARCO_OK;
 }
 
-int varco_launch_compress_slots(const varco_plan *pl, const void *Gh, int64_t ld, int F, int k, varco_dtype_t dt,
-                                varco_key_t key, void *packed, int64_t kstride, cudaStream_t st) {
+// packed rows (slot order, stride kstride) -> (value, position) pairs, pstride pairs per slot
+int varco_launch_expand_slots(const varco_plan *pl, const void *packed, int64_t kstride, int F, int k,
+                              varco_dtype_t dt, varco_key_t key, void *pairs, int64_t pstride, cudaStream_t st) {
   if (pl->H == 0) return VARCO_OK;
-  const int es = dt == VARCO_F32 ? 4 : 2, V = 16 / es;
-  const int nv = (F + V - 1) / V, kv = (k + V - 1) / V;
-  HaloLaunch L = shape(pl->H, nv, (size_t)(nv + kv) * 16);
+  const int G = k <= 8 ? 8 : (k <= 16 ? 16 : 32);
   const int h = vperm::half_bits(F);
   const uint64_t lkey = vperm::layer_key(key);
+  const int threads = 256;
+  const unsigned blocks = (unsigned)(((int64_t)pl->H * G + threads - 1) / threads);
+  HaloLaunch L;
+  L.G = G;
   if (dt == VARCO_F32)
-    VARCO_DISPATCH_G(L, (compress_slots_kernel<uint32_t, G><<<L.blocks, L.threads, L.smem, st>>>(
-                            (const uint32_t *)Gh, ld, F, k, h, lkey, pl->d.slot_gid, (int)pl->H, (uint32_t *)packed,
-                            kstride)));
+    VARCO_DISPATCH_G(L, (expand_slots_kernel<uint32_t, G><<<blocks, threads, 0, st>>>(
+                            (const uint32_t *)packed, kstride, F, k, h, lkey, pl->d.slot_gid, (int)pl->H,
+                            (uint32_t *)pairs, pstride)));
   else
-    VARCO_DISPATCH_G(L, (compress_slots_kernel<uint16_t, G><<<L.blocks, L.threads, L.smem, st>>>(
-                            (const uint16_t *)Gh, ld, F, k, h, lkey, pl->d.slot_gid, (int)pl->H, (uint16_t *)packed,
-                            kstride)));
+    VARCO_DISPATCH_G(L, (expand_slots_kernel<uint16_t, G><<<blocks, threads, 0, st>>>(
+                            (const uint16_t *)packed, kstride, F, k, h, lkey, pl->d.slot_gid, (int)pl->H,
+                            (uint32_t *)pairs, pstride)));
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }

@@ -21,8 +21,8 @@ int varco_launch_compress_rows(const varco_plan *pl, const void *X, int64_t ld, 
                                varco_key_t key, void *packed, int64_t kstride, int send_order, cudaStream_t st);
 int varco_launch_decompress_slots(const varco_plan *pl, const void *packed, int64_t kstride, int send_order, int F,
                                   int k, varco_dtype_t dt, varco_key_t key, void *Xhalo, int64_t ld, cudaStream_t st);
-int varco_launch_compress_slots(const varco_plan *pl, const void *Gh, int64_t ld, int F, int k, varco_dtype_t dt,
-                                varco_key_t key, void *packed, int64_t kstride, cudaStream_t st);
+int varco_launch_expand_slots(const varco_plan *pl, const void *packed, int64_t kstride, int F, int k,
+                              varco_dtype_t dt, varco_key_t key, void *pairs, int64_t pstride, cudaStream_t st);
 int varco_launch_scatter_add_rows(const varco_plan *pl, const void *packed, int64_t kstride, int F, int k,
                                   varco_dtype_t dt, varco_key_t key, void *dX, int64_t ld, cudaStream_t st);
 int varco_launch_add_dense_rows(const varco_plan *pl, const void *Gh, int64_t ldg, int F, varco_dtype_t dt, void *dX,
@@ -31,7 +31,11 @@ int varco_launch_add_dense_rows(const varco_plan *pl, const void *Gh, int64_t ld
 int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, const void *Xhalo, int64_t ldh, int F,
                           varco_dtype_t dt, void *Agg, int64_t ldagg, cudaStream_t st);
 int varco_launch_spmm_bwd(const varco_plan *pl, const void *dAgg, int64_t ldd, int F, varco_dtype_t dt, void *dX,
-                          int64_t ldx, int accumulate, void *Ghalo, int64_t ldh, cudaStream_t st);
+                          int64_t ldx, int accumulate, void *Ghalo, int64_t ldh, void *packed, int64_t kstride, int k,
+                          varco_key_t key, cudaStream_t st);
+int varco_launch_spmm_fwd_sparse(const varco_plan *pl, const void *X, int64_t ldx, const void *pairs, int64_t pstride,
+                                 int k, int F, varco_dtype_t dt, void *Agg, int64_t ldagg, cudaStream_t st);
+bool varco_spmm_sparse_supported(int F, int k, varco_dtype_t dt);
 // gemm_simt.cu
 size_t varco_simt_dw_scratch_bytes(int F_in, int F_out);
 int varco_simt_gemm_fwd(int n, int F_in, int F_out, varco_dtype_t dt, const void *X, int64_t ldx, const void *Agg,

@@ -103,6 +103,10 @@ int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   // receiver, so "send buffer -> receive buffer" is folded into the write address.  At full
   // communication the row travels whole and in order: one gather-copy fills the halo slots.
   const int64_t kstride = round_up64(k, V);
+  // Compressed epochs with at most a quarter of a row kept: the receiver keeps (value, position)
+  // pairs instead of rows that are mostly zeros, and the aggregation reads k pairs per remote
+  // neighbour instead of F elements.
+  const bool sparse = k < F_in && varco_spmm_sparse_supported(F_in, k, dt);
   if (k == F_in) {
     StageTimer t(plan, VARCO_STAGE_COMPRESS, stream);
     rc = varco_launch_gather_copy(plan, X, desc->ld_in, F_in, dt, Xhalo, L.ld_in, st);
@@ -113,12 +117,19 @@ int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
     }
     if (rc != VARCO_OK) return rc;
     StageTimer t(plan, VARCO_STAGE_DECOMPRESS, stream);
-    rc = varco_launch_decompress_slots(plan, packed, kstride, 0, F_in, k, dt, key, Xhalo, L.ld_in, st);
+    if (sparse)
+      rc = varco_launch_expand_slots(plan, packed, kstride, F_in, k, dt, key, Xhalo, round_up64(k, 4), st);
+    else
+      rc = varco_launch_decompress_slots(plan, packed, kstride, 0, F_in, k, dt, key, Xhalo, L.ld_in, st);
   }
   if (rc != VARCO_OK) return rc;
   {
     StageTimer t(plan, VARCO_STAGE_SPMM, stream);
-    rc = varco_launch_spmm_fwd(plan, X, desc->ld_in, Xhalo, L.ld_in, F_in, dt, Agg_saved, desc->ld_in, st);
+    if (sparse)
+      rc = varco_launch_spmm_fwd_sparse(plan, X, desc->ld_in, Xhalo, round_up64(k, 4), k, F_in, dt, Agg_saved,
+                                        desc->ld_in, st);
+    else
+      rc = varco_launch_spmm_fwd(plan, X, desc->ld_in, Xhalo, L.ld_in, F_in, dt, Agg_saved, desc->ld_in, st);
   }
   if (rc != VARCO_OK) return rc;
   {
@@ -213,7 +224,9 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   if (rc != VARCO_OK) return rc;
   {
     StageTimer t(plan, VARCO_STAGE_SPMM_T, stream);
-    rc = varco_launch_spmm_bwd(plan, dAgg, L.ld_in, F_in, dt, dX, desc->ld_in, sage ? 1 : 0, Ghalo, L.ld_in, st);
+    // k < F: the slot gradients are compressed in the epilogue (no dense slot rows)
+    rc = varco_launch_spmm_bwd(plan, dAgg, L.ld_in, F_in, dt, dX, desc->ld_in, sage ? 1 : 0, Ghalo, L.ld_in,
+                               k < F_in ? packed : nullptr, round_up64(k, V), k, key, st);
   }
   if (rc != VARCO_OK) return rc;
   // Return of the halo-slot gradients to the owners.  At full communication the slot rows are
@@ -223,11 +236,6 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
     return varco_launch_add_dense_rows(plan, Ghalo, L.ld_in, F_in, dt, dX, desc->ld_in, st);
   }
   const int64_t kstride = round_up64(k, V);
-  {
-    StageTimer t(plan, VARCO_STAGE_COMPRESS_BWD, stream);
-    rc = varco_launch_compress_slots(plan, Ghalo, L.ld_in, F_in, k, dt, key, packed, kstride, st);
-  }
-  if (rc != VARCO_OK) return rc;
   {
     StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
     rc = varco_launch_scatter_add_rows(plan, packed, kstride, F_in, k, dt, key, dX, desc->ld_in, st);

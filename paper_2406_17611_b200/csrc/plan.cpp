@@ -181,6 +181,14 @@ int build(varco_plan *pl, int64_t n, const int64_t *rp0, const int32_t *col0, co
     }
   });
 
+  // number of leading entries of every row whose source is a local row (columns are sorted: local first)
+  pl->nloc.resize(n);
+  for (int64_t r = 0; r < n; ++r) {
+    int32_t c = 0;
+    for (int64_t e = pl->rp[r]; e < pl->rp[r + 1] && pl->col[e] < n; ++e) ++c;
+    pl->nloc[r] = c;
+  }
+
   // transpose: sources [0, n + H) -> the rows that use them (ascending row inside a source)
   const int64_t nsrc = n + pl->H;
   pl->rpT.assign(nsrc + 1, 0);

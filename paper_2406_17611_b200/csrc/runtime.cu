@@ -22,6 +22,7 @@ std::vector<ImageItem> image_items(varco_plan *pl) {
   varco_dev_image &d = pl->d;
   return {item(pl->row_gid, &d.row_gid),
           item(pl->rp, &d.rp),
+          item(pl->nloc, &d.nloc),
           item(pl->col, &d.col),
           item(pl->val, &d.val),
           item(pl->rpT, &d.rpT),

@@ -30,6 +30,16 @@ struct RowClass {
   int count;
 };
 
+// Optional epilogue of the transposed pass: a halo-slot gradient row is not written out densely but
+// compressed on the spot with the forward's key (k values at the kept positions, slot order).
+struct HaloCompress {
+  void *packed;          // nullptr: write dense rows
+  int64_t kstride;       // elements per packed row
+  int k, F, h;
+  uint64_t lkey;
+  const int32_t *slot_gid;
+};
+
 struct SpmmArgs {
   const int64_t *rp;
   const int32_t *col;
@@ -50,6 +60,7 @@ struct SpmmArgs {
   int nv;        // 16-byte chunks per row
   int panels;    // feature panels
   int nv_panel;  // chunks per panel
+  HaloCompress hc;
 };
 
 // task id -> (position in the class list, panel); tasks are ordered (partition, panel, row)
@@ -135,7 +146,8 @@ template <typename T, int G, int NCH, int UNR, bool FULL>
 __global__ void __launch_bounds__(256)
     spmm_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col, const float *__restrict__ val,
                 RowClass rc, int P, int panels, int nv_panel, GatherSrc gs, T *__restrict__ O0, int64_t ldo0,
-                T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv) {
+                T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv, HaloCompress hc) {
+  extern __shared__ uint4 stage_rows[];
   constexpr int V = ElemTraits<T>::kVec;
   const int64_t task = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
   const int gl = threadIdx.x % G;
@@ -155,6 +167,25 @@ __global__ void __launch_bounds__(256)
     for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
   const int64_t e0 = rp[r];
   accumulate_range<T, G, NCH, UNR, FULL>(col + e0, val + e0, (int)(rp[r + 1] - e0), gs, ch_lo, ch_hi, gl, gmask, acc);
+  if (hc.packed && r >= dst_split) {
+    // stage the row in the element type, pick the kept positions, write k values
+    typedef typename ElemBits<T>::type E;
+    uint4 *srow4 = stage_rows + (size_t)(threadIdx.x / G) * nv;
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+      const int ch = gl + i * G;
+      if (FULL || ch < nv) srow4[ch] = pack16(acc[i], T());
+    }
+    const int slot = r - dst_split;
+    vperm::RowPerm pm;
+    if (G >= 8) init_perm<(G >= 8 ? G : 8)>(pm, hc.lkey, (uint32_t)__ldg(hc.slot_gid + slot), (uint32_t)hc.F, hc.h, gl, gmask);
+    else pm.init(hc.lkey, (uint32_t)__ldg(hc.slot_gid + slot), (uint32_t)hc.F, hc.h);
+    __syncwarp(gmask);
+    const E *srow = reinterpret_cast<const E *>(srow4);
+    E *z = reinterpret_cast<E *>(hc.packed) + (int64_t)slot * hc.kstride;
+    for (int m = gl; m < (int)hc.kstride; m += G) z[m] = m < hc.k ? srow[pm.pi((uint32_t)m)] : (E)0;
+    return;
+  }
   bool add;
   uint4 *dst = dest_row<T>(r, O0, ldo0, O1, ldo1, dst_split, accumulate0, add);
 #pragma unroll
@@ -178,7 +209,7 @@ template <typename T, int NCH, int UNR, bool FULL>
 __global__ void __launch_bounds__(256)
     spmm_hub_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col, const float *__restrict__ val,
                     RowClass rc, int P, int panels, int nv_panel, GatherSrc gs, T *__restrict__ O0, int64_t ldo0,
-                    T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv) {
+                    T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv, HaloCompress hc) {
   extern __shared__ float hub_part[];
   constexpr int V = ElemTraits<T>::kVec;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
@@ -209,6 +240,33 @@ __global__ void __launch_bounds__(256)
       for (int j = 0; j < V; ++j) hub_part[(size_t)warp * row_floats + c * V + j] = acc[i][j];
   }
   __syncthreads();
+  if (hc.packed && r >= dst_split) {
+    // reduce into the first warp's row, convert in place to the element type, then compress
+    typedef typename ElemBits<T>::type E;
+    uint4 *srow4 = reinterpret_cast<uint4 *>(hub_part);
+    uint4 mine[(NCH * 32 + 255) / 256 + 1];
+    int cnt = 0;
+    for (int c = threadIdx.x; c < nv; c += blockDim.x) {
+      float f[V];
+#pragma unroll
+      for (int j = 0; j < V; ++j) f[j] = 0.f;
+      for (int w = 0; w < nwarps; ++w)
+#pragma unroll
+        for (int j = 0; j < V; ++j) f[j] += hub_part[(size_t)w * row_floats + c * V + j];
+      mine[cnt++] = pack16(f, T());
+    }
+    __syncthreads();
+    cnt = 0;
+    for (int c = threadIdx.x; c < nv; c += blockDim.x) srow4[c] = mine[cnt++];
+    __syncthreads();
+    const int slot = r - dst_split;
+    vperm::RowPerm pm;
+    pm.init(hc.lkey, (uint32_t)__ldg(hc.slot_gid + slot), (uint32_t)hc.F, hc.h);
+    const E *srow = reinterpret_cast<const E *>(srow4);
+    E *z = reinterpret_cast<E *>(hc.packed) + (int64_t)slot * hc.kstride;
+    for (int m = threadIdx.x; m < (int)hc.kstride; m += blockDim.x) z[m] = m < hc.k ? srow[pm.pi((uint32_t)m)] : (E)0;
+    return;
+  }
   bool add;
   uint4 *dst = dest_row<T>(r, O0, ldo0, O1, ldo1, dst_split, accumulate0, add);
   for (int c = threadIdx.x; c < ch_hi - ch_lo; c += blockDim.x) {
@@ -246,11 +304,11 @@ int launch_hubs(const SpmmArgs &a, cudaStream_t st) {
   if (a.panels == 1 && a.nv == 32 * NCH)
     spmm_hub_kernel<T, NCH, UNR, true><<<grid, warps * 32, warps * row_bytes, st>>>(
         a.rp, a.col, a.val, a.hubs, a.P, a.panels, a.nv_panel, gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1,
-        a.dst_split, a.accumulate0, a.nv);
+        a.dst_split, a.accumulate0, a.nv, a.hc);
   else
     spmm_hub_kernel<T, NCH, UNR, false><<<grid, warps * 32, warps * row_bytes, st>>>(
         a.rp, a.col, a.val, a.hubs, a.P, a.panels, a.nv_panel, gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1,
-        a.dst_split, a.accumulate0, a.nv);
+        a.dst_split, a.accumulate0, a.nv, a.hc);
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
@@ -261,14 +319,15 @@ int launch_rows(const SpmmArgs &a, const RowClass &rc, cudaStream_t st) {
   const int threads = 256;
   const int64_t total = (int64_t)rc.count * a.panels * G;
   dim3 grid((unsigned)((total + threads - 1) / threads));
+  const size_t smem = a.hc.packed ? (size_t)(threads / G) * a.nv * 16 : 0;
   if (a.panels == 1 && a.nv == G * NCH)
-    spmm_kernel<T, G, NCH, UNR, true><<<grid, threads, 0, st>>>(a.rp, a.col, a.val, rc, a.P, a.panels, a.nv_panel,
-                                                                gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1,
-                                                                a.dst_split, a.accumulate0, a.nv);
+    spmm_kernel<T, G, NCH, UNR, true><<<grid, threads, smem, st>>>(a.rp, a.col, a.val, rc, a.P, a.panels, a.nv_panel,
+                                                                   gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1,
+                                                                   a.ldo1, a.dst_split, a.accumulate0, a.nv, a.hc);
   else
-    spmm_kernel<T, G, NCH, UNR, false><<<grid, threads, 0, st>>>(a.rp, a.col, a.val, rc, a.P, a.panels, a.nv_panel,
-                                                                 gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1,
-                                                                 a.ldo1, a.dst_split, a.accumulate0, a.nv);
+    spmm_kernel<T, G, NCH, UNR, false><<<grid, threads, smem, st>>>(a.rp, a.col, a.val, rc, a.P, a.panels, a.nv_panel,
+                                                                    gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1,
+                                                                    a.ldo1, a.dst_split, a.accumulate0, a.nv, a.hc);
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
@@ -295,6 +354,224 @@ int dispatch(const SpmmArgs &a, cudaStream_t st) {
   if (w <= 96) return launch<T, 32, 3, 4, 16, 6, 1>(a, st);
   if (w <= 128) return launch<T, 32, 4, 2, 32, 4, 1>(a, st);
   if (w <= 256) return launch<T, 32, 8, 2, 32, 8, 1>(a, st);
+  return VARCO_UNSUPPORTED;
+}
+
+// ------------------------------------------------------------------------------------------
+// Forward aggregation with SPARSE halo rows (compressed epochs).  A remote neighbour contributes
+// only its k kept values, so its slot is stored as k (value, position) pairs and the row's
+// remote part is accumulated by scattering those pairs into a shared-memory fp32 row; the local
+// part goes through the dense register path above.  Entry order is unchanged (local entries
+// first, then halo slots ascending).
+template <typename T> struct SparsePair;
+template <> struct SparsePair<float> {
+  typedef uint2 type;
+  __device__ static __forceinline__ float val(uint2 p) { return __uint_as_float(p.x); }
+  __device__ static __forceinline__ int pos(uint2 p) { return (int)p.y; }
+};
+template <> struct SparsePair<__nv_bfloat16> {
+  typedef uint32_t type;
+  __device__ static __forceinline__ float val(uint32_t p) { return __uint_as_float(p << 16); }
+  __device__ static __forceinline__ int pos(uint32_t p) { return (int)(p >> 16); }
+};
+
+// halo entries [0, len) of one row: sacc[pos] += w * value for the k pairs of every entry's slot
+template <typename T, int G>
+__device__ __forceinline__ void accumulate_sparse(const int32_t *__restrict__ colp, const float *__restrict__ valp,
+                                                  int len, const typename SparsePair<T>::type *__restrict__ pairs,
+                                                  int64_t pstride, int k, int split, float *sacc, int gl,
+                                                  unsigned gmask) {
+  typedef typename SparsePair<T>::type P;
+  for (int base = 0; base < len; base += G) {
+    const int cnt = min(G, len - base);
+    const int mine = base + min(gl, cnt - 1);
+    const int myc = __ldg(colp + mine);
+    const float myw = gl < cnt ? __ldg(valp + mine) : 0.f;
+    if (k <= G) {
+      // one pair per lane and entry: fetch four entries ahead of the shared-memory updates
+      for (int t = 0; t < cnt; t += 4) {
+        P p[4];
+        float w[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int slot = __shfl_sync(gmask, myc, t + u, G) - split;
+          w[u] = __shfl_sync(gmask, myw, t + u, G);
+          p[u] = __ldg(pairs + (int64_t)slot * pstride + min(gl, k - 1));
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (gl < k) sacc[SparsePair<T>::pos(p[u])] += w[u] * SparsePair<T>::val(p[u]);
+          __syncwarp(gmask);
+        }
+      }
+    } else {
+      for (int t = 0; t < cnt; ++t) {
+        const int slot = __shfl_sync(gmask, myc, t, G) - split;
+        const float w = __shfl_sync(gmask, myw, t, G);
+        const P *pr = pairs + (int64_t)slot * pstride;
+        for (int m = gl; m < k; m += G) {
+          const P q = __ldg(pr + m);
+          sacc[SparsePair<T>::pos(q)] += w * SparsePair<T>::val(q);
+        }
+        __syncwarp(gmask);
+      }
+    }
+  }
+}
+
+// One group per row (normal and short classes).  Shared memory: F floats per group.
+template <typename T, int G, int NCH, bool FULL>
+__global__ void __launch_bounds__(256)
+    spmm_sparse_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ nloc,
+                       const int32_t *__restrict__ col, const float *__restrict__ val, RowClass rc, GatherSrc gs,
+                       const typename SparsePair<T>::type *__restrict__ pairs, int64_t pstride, int k,
+                       T *__restrict__ O, int64_t ldo, int nv) {
+  extern __shared__ float sparse_acc[];
+  constexpr int V = ElemTraits<T>::kVec;
+  const int task = (blockIdx.x * blockDim.x + threadIdx.x) / G;
+  const int grp = threadIdx.x / G, gl = threadIdx.x % G;
+  const unsigned lane = threadIdx.x % 32;
+  const unsigned gmask = (G == 32) ? 0xFFFFFFFFu : (((1u << G) - 1u) << (lane & ~(unsigned)(G - 1)));
+  float *sacc = sparse_acc + (size_t)grp * nv * V;
+  if (task >= rc.count) return;
+  for (int c = gl; c < nv * V; c += G) sacc[c] = 0.f;
+  const int r = __ldg(rc.rows + task);
+  const int64_t e0 = rp[r];
+  const int len = (int)(rp[r + 1] - e0);
+  const int nl = __ldg(nloc + r);
+  float acc[NCH][V];
+#pragma unroll
+  for (int i = 0; i < NCH; ++i)
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
+  __syncwarp(gmask);
+  if (nl > 0) accumulate_range<T, G, NCH, 4, FULL>(col + e0, val + e0, nl, gs, 0, nv, gl, gmask, acc);
+  if (len > nl) accumulate_sparse<T, G>(col + e0 + nl, val + e0 + nl, len - nl, pairs, pstride, k, gs.split, sacc, gl, gmask);
+  uint4 *dst = reinterpret_cast<uint4 *>(O + (int64_t)r * ldo);
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    const int ch = gl + i * G;
+    if (FULL || ch < nv) {
+#pragma unroll
+      for (int j = 0; j < V; ++j) acc[i][j] += sacc[ch * V + j];
+      dst[ch] = pack16(acc[i], T());
+    }
+  }
+}
+
+// Hubs: one CTA per row; every warp takes a contiguous share of the local and of the halo entries and
+// owns one shared-memory row; the rows are added in warp order.
+template <typename T, int NCH, bool FULL>
+__global__ void __launch_bounds__(256)
+    spmm_sparse_hub_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ nloc,
+                           const int32_t *__restrict__ col, const float *__restrict__ val, RowClass rc, GatherSrc gs,
+                           const typename SparsePair<T>::type *__restrict__ pairs, int64_t pstride, int k,
+                           T *__restrict__ O, int64_t ldo, int nv) {
+  extern __shared__ float sparse_acc[];
+  constexpr int V = ElemTraits<T>::kVec;
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int nwarps = blockDim.x / 32;
+  const int rowf = nv * V;
+  float *sacc = sparse_acc + (size_t)warp * rowf;
+  for (int c = lane; c < rowf; c += 32) sacc[c] = 0.f;
+  const int r = __ldg(rc.rows + blockIdx.x);
+  const int64_t e0 = rp[r];
+  const int len = (int)(rp[r + 1] - e0);
+  const int nl = __ldg(nloc + r);
+  float acc[NCH][V];
+#pragma unroll
+  for (int i = 0; i < NCH; ++i)
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
+  __syncwarp();
+  auto share = [&](int total, int &b0, int &b1) {
+    const int per = ((total + nwarps - 1) / nwarps + 31) / 32 * 32;
+    b0 = min(total, warp * per);
+    b1 = min(total, b0 + per);
+  };
+  int b0, b1;
+  share(nl, b0, b1);
+  if (b1 > b0) accumulate_range<T, 32, NCH, 4, FULL>(col + e0 + b0, val + e0 + b0, b1 - b0, gs, 0, nv, lane, 0xFFFFFFFFu, acc);
+  share(len - nl, b0, b1);
+  if (b1 > b0)
+    accumulate_sparse<T, 32>(col + e0 + nl + b0, val + e0 + nl + b0, b1 - b0, pairs, pstride, k, gs.split, sacc, lane,
+                             0xFFFFFFFFu);
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    const int ch = lane + i * 32;
+    if (FULL || ch < nv)
+#pragma unroll
+      for (int j = 0; j < V; ++j) sacc[ch * V + j] += acc[i][j];
+  }
+  __syncthreads();
+  uint4 *dst = reinterpret_cast<uint4 *>(O + (int64_t)r * ldo);
+  for (int ch = threadIdx.x; ch < nv; ch += blockDim.x) {
+    float f[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) f[j] = 0.f;
+    for (int w = 0; w < nwarps; ++w)
+#pragma unroll
+      for (int j = 0; j < V; ++j) f[j] += sparse_acc[(size_t)w * rowf + ch * V + j];
+    dst[ch] = pack16(f, T());
+  }
+}
+
+template <typename T, int G, int NCH>
+int launch_sparse_rows(const SpmmArgs &a, const RowClass &rc, const int32_t *nloc, const void *pairs, int64_t pstride,
+                       int k, cudaStream_t st) {
+  if (rc.count == 0) return VARCO_OK;
+  constexpr int V = ElemTraits<T>::kVec;
+  typedef typename SparsePair<T>::type P;
+  const int threads = 256;
+  const size_t smem = (size_t)(threads / G) * a.nv * V * sizeof(float);
+  dim3 grid((unsigned)(((int64_t)rc.count * G + threads - 1) / threads));
+  if (a.nv == G * NCH)
+    spmm_sparse_kernel<T, G, NCH, true><<<grid, threads, smem, st>>>(a.rp, nloc, a.col, a.val, rc, gather_src<T>(a),
+                                                                     (const P *)pairs, pstride, k, (T *)a.O0, a.ldo0,
+                                                                     a.nv);
+  else
+    spmm_sparse_kernel<T, G, NCH, false><<<grid, threads, smem, st>>>(a.rp, nloc, a.col, a.val, rc, gather_src<T>(a),
+                                                                      (const P *)pairs, pstride, k, (T *)a.O0, a.ldo0,
+                                                                      a.nv);
+  VARCO_KERNEL_LAUNCHED();
+  return VARCO_OK;
+}
+
+template <typename T, int NCH>
+int launch_sparse_hubs(const SpmmArgs &a, const int32_t *nloc, const void *pairs, int64_t pstride, int k,
+                       cudaStream_t st) {
+  if (a.hubs.count == 0) return VARCO_OK;
+  constexpr int V = ElemTraits<T>::kVec;
+  typedef typename SparsePair<T>::type P;
+  const size_t row_bytes = (size_t)a.nv * V * sizeof(float);
+  int warps = 8;
+  while (warps > 1 && warps * row_bytes > 48 * 1024) warps /= 2;
+  if (a.nv == 32 * NCH)
+    spmm_sparse_hub_kernel<T, NCH, true><<<a.hubs.count, warps * 32, warps * row_bytes, st>>>(
+        a.rp, nloc, a.col, a.val, a.hubs, gather_src<T>(a), (const P *)pairs, pstride, k, (T *)a.O0, a.ldo0, a.nv);
+  else
+    spmm_sparse_hub_kernel<T, NCH, false><<<a.hubs.count, warps * 32, warps * row_bytes, st>>>(
+        a.rp, nloc, a.col, a.val, a.hubs, gather_src<T>(a), (const P *)pairs, pstride, k, (T *)a.O0, a.ldo0, a.nv);
+  VARCO_KERNEL_LAUNCHED();
+  return VARCO_OK;
+}
+
+// lanes per row for the ordinary class / the short class, by row width in chunks (nv <= 64 only)
+template <typename T>
+int dispatch_sparse(const SpmmArgs &a, const int32_t *nloc, const void *pairs, int64_t pstride, int k,
+                    cudaStream_t st) {
+  const int w = a.nv;
+#define VARCO_SPARSE(G, NCH, GS, NCHS)                                                               \
+  do {                                                                                               \
+    if (int rc = launch_sparse_hubs<T, (NCH * G + 31) / 32>(a, nloc, pairs, pstride, k, st)) return rc; \
+    if (int rc = launch_sparse_rows<T, G, NCH>(a, a.normal, nloc, pairs, pstride, k, st)) return rc;  \
+    return launch_sparse_rows<T, GS, NCHS>(a, a.shorts, nloc, pairs, pstride, k, st);                 \
+  } while (0)
+  if (w <= 8) VARCO_SPARSE(8, 1, 8, 1);
+  if (w <= 16) VARCO_SPARSE(16, 1, 8, 2);
+  if (w <= 32) VARCO_SPARSE(32, 1, 8, 4);
+  if (w <= 64) VARCO_SPARSE(32, 2, 16, 4);
+#undef VARCO_SPARSE
   return VARCO_UNSUPPORTED;
 }
 
@@ -330,12 +607,50 @@ int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, cons
   return dt == VARCO_F32 ? dispatch<float>(a, st) : dispatch<__nv_bfloat16>(a, st);
 }
 
+bool varco_spmm_sparse_supported(int F, int k, varco_dtype_t dt) {
+  const int V = dt == VARCO_F32 ? 4 : 8;
+  const int nv = (F + V - 1) / V;
+  // pays (measured) when a remote row shrinks to at most an eighth; positions must fit the pair format;
+  // 32 groups of nv * V floats must fit the default shared-memory window
+  return nv <= 64 && 8 * k <= F && F <= 65535 && (size_t)32 * nv * V * sizeof(float) <= 48 * 1024;
+}
+
+// Forward aggregation when the halo slots hold (value, position) pairs instead of dense rows.
+int varco_launch_spmm_fwd_sparse(const varco_plan *pl, const void *X, int64_t ldx, const void *pairs, int64_t pstride,
+                                 int k, int F, varco_dtype_t dt, void *Agg, int64_t ldagg, cudaStream_t st) {
+  const int V = dt == VARCO_F32 ? 4 : 8;
+  SpmmArgs a{};
+  a.rp = pl->d.rp;
+  a.col = pl->d.col;
+  a.val = pl->d.val;
+  a.hubs = RowClass{pl->d.hub_f, pl->d.hub_f_start, (int)pl->hub_f.size()};
+  a.normal = RowClass{pl->d.order_f, pl->d.order_f_start, (int)pl->order_f.size()};
+  a.shorts = RowClass{pl->d.short_f, pl->d.short_f_start, (int)pl->short_f.size()};
+  a.P = pl->P;
+  a.A0 = X;
+  a.lda0 = ldx;
+  a.A1 = X;
+  a.lda1 = ldx;
+  a.src_split = (int)pl->n;
+  a.O0 = Agg;
+  a.ldo0 = ldagg;
+  a.dst_split = (int)pl->n;
+  a.nv = (F + V - 1) / V;
+  a.panels = 1;
+  a.nv_panel = a.nv;
+  return dt == VARCO_F32 ? dispatch_sparse<float>(a, pl->d.nloc, pairs, pstride, k, st)
+                         : dispatch_sparse<__nv_bfloat16>(a, pl->d.nloc, pairs, pstride, k, st);
+}
+
 // Transposed aggregation: for a source u, g_u = sum over the rows i that use it of s_iu dAgg[i];
 // u < n lands in dX[u] (added to what is there when `accumulate`), u >= n in Ghalo[u - n].
 // Every source of partition q is used by rows of q only, so the gathered set of a partition is
 // its own block of dAgg: panels are chosen so that this block stays in L2.
+// With `packed` set (k < F) the halo-slot rows are compressed in the kernels' epilogue with the forward's
+// key and only the k kept values of every slot are written (slot order, stride kstride).
 int varco_launch_spmm_bwd(const varco_plan *pl, const void *dAgg, int64_t ldd, int F, varco_dtype_t dt, void *dX,
-                          int64_t ldx, int accumulate, void *Ghalo, int64_t ldh, cudaStream_t st) {
+                          int64_t ldx, int accumulate, void *Ghalo, int64_t ldh, void *packed, int64_t kstride, int k,
+                          varco_key_t key, cudaStream_t st) {
   const int V = dt == VARCO_F32 ? 4 : 8;
   const int nv = (F + V - 1) / V;
   SpmmArgs a{};
@@ -360,5 +675,6 @@ int varco_launch_spmm_bwd(const varco_plan *pl, const void *dAgg, int64_t ldd, i
   a.nv = nv;
   a.panels = 1;
   a.nv_panel = nv;
+  if (packed) a.hc = HaloCompress{packed, kstride, k, F, vperm::half_bits(F), vperm::layer_key(key), pl->d.slot_gid};
   return dt == VARCO_F32 ? dispatch<float>(a, st) : dispatch<__nv_bfloat16>(a, st);
 }

@@ -14,6 +14,7 @@ struct varco_dev_image {
   // aggregation structure of all partitions: row r aggregates from sources col[e] with weight
   // val[e]; a source < n is the local row of X with that index, a source >= n is halo slot (col - n)
   const int64_t *rp = nullptr;
+  const int32_t *nloc = nullptr;   // leading entries of a forward row that point at local rows
   const int32_t *col = nullptr;
   const float *val = nullptr;
   // transposed structure: source u (row or n + slot) is used by rows colT[e] with weight valT[e]
@@ -50,7 +51,7 @@ struct varco_plan {
   std::vector<int64_t> new_to_old, part_off, counts, send_base, halo_ids;
   // host copies of the device image
   std::vector<int32_t> row_gid, col, colT, slot_gid, slot_src, slot_sendpos, brow, brow_ptr, brow_slot;
-  std::vector<int32_t> order_f, order_t, hub_f, hub_t, short_f, short_t;
+  std::vector<int32_t> order_f, order_t, hub_f, hub_t, short_f, short_t, nloc;
   std::vector<int32_t> order_f_start, order_t_start, hub_f_start, hub_t_start, short_f_start, short_t_start;
   std::vector<int64_t> rp, rpT;
   std::vector<float> val, valT;
