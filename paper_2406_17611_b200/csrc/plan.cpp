@@ -230,7 +230,7 @@ int build(varco_plan *pl, int64_t n, const int64_t *rp0, const int32_t *col0, co
   // rows per warp.  The rest get a full-width group.  Every class list is partition-major (the
   // kernels sweep partition by partition so that a partition's gathered rows stay in L2) and, inside
   // a partition, sorted by length, longest first, so that the lanes of a warp run alike.
-  const int64_t kHubEntries = 512, kShortEntries = 8;
+  const int64_t kHubEntries = 512, kShortEntries = 8;   // the record format below holds 8 entries
   auto classify = [&](const std::vector<int64_t> &ptr, const std::vector<std::vector<int32_t>> &rows_of_part,
                       std::vector<int32_t> *lists[3], std::vector<int32_t> *starts[3]) {
     for (int c = 0; c < 3; ++c) {
@@ -265,6 +265,23 @@ int build(varco_plan *pl, int64_t n, const int64_t *rp0, const int32_t *col0, co
     std::vector<int32_t> *stt[3] = {&pl->hub_t_start, &pl->order_t_start, &pl->short_t_start};
     classify(pl->rpT, rows_of_part, lt, stt);
   }
+  // fixed-size records of the short rows, in class-list order: 8 sources and 8 weights per row
+  // (-1 / 0 beyond the row's length).  The short-row kernels find them by thread index alone, so
+  // the gathers start after ONE dependent load instead of three (row id -> row_ptr -> columns).
+  auto records = [&](const std::vector<int64_t> &ptr, const std::vector<int32_t> &cols, const std::vector<float> &vals,
+                     const std::vector<int32_t> &rows, std::vector<int32_t> &rec_col, std::vector<float> &rec_val) {
+    rec_col.assign(rows.size() * 8, -1);
+    rec_val.assign(rows.size() * 8, 0.f);
+    for (size_t i = 0; i < rows.size(); ++i) {
+      const int64_t e0 = ptr[rows[i]], len = ptr[rows[i] + 1] - e0;
+      for (int64_t j = 0; j < len; ++j) {
+        rec_col[i * 8 + j] = cols[e0 + j];
+        rec_val[i * 8 + j] = vals[e0 + j];
+      }
+    }
+  };
+  records(pl->rp, pl->col, pl->val, pl->short_f, pl->short_f_col, pl->short_f_val);
+  records(pl->rpT, pl->colT, pl->valT, pl->short_t, pl->short_t_col, pl->short_t_val);
   return VARCO_OK;
 }
 

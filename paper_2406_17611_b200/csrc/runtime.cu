@@ -40,6 +40,10 @@ std::vector<ImageItem> image_items(varco_plan *pl) {
           item(pl->hub_t, &d.hub_t),
           item(pl->short_f, &d.short_f),
           item(pl->short_t, &d.short_t),
+          item(pl->short_f_col, &d.short_f_col),
+          item(pl->short_t_col, &d.short_t_col),
+          item(pl->short_f_val, &d.short_f_val),
+          item(pl->short_t_val, &d.short_t_val),
           item(pl->order_f_start, &d.order_f_start),
           item(pl->order_t_start, &d.order_t_start),
           item(pl->hub_f_start, &d.hub_f_start),

@@ -22,6 +22,10 @@
 #include "device_common.cuh"
 #include "kernels.h"
 
+#ifndef VARCO_SHORT_UNR
+#define VARCO_SHORT_UNR 2
+#endif
+
 namespace {
 
 struct RowClass {
@@ -61,6 +65,8 @@ struct SpmmArgs {
   int panels;    // feature panels
   int nv_panel;  // chunks per panel
   HaloCompress hc;
+  const int32_t *short_col;   // 8-entry records of the short class (nullptr: walk the CSR)
+  const float *short_val;
 };
 
 // task id -> (position in the class list, panel); tasks are ordered (partition, panel, row)
@@ -142,31 +148,14 @@ __device__ __forceinline__ uint4 *dest_row(int r, T *O0, int64_t ldo0, T *O1, in
   return reinterpret_cast<uint4 *>(O1 + (int64_t)(r - dst_split) * ldo1);
 }
 
-template <typename T, int G, int NCH, int UNR, bool FULL>
-__global__ void __launch_bounds__(256)
-    spmm_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col, const float *__restrict__ val,
-                RowClass rc, int P, int panels, int nv_panel, GatherSrc gs, T *__restrict__ O0, int64_t ldo0,
-                T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv, HaloCompress hc) {
-  extern __shared__ uint4 stage_rows[];
+// Write one finished row: dense (optionally added to what is there), or -- for a halo-slot gradient row of
+// the transposed pass when hc.packed is set -- compressed with the forward's key.
+template <typename T, int G, int NCH, bool FULL>
+__device__ __forceinline__ void finish_row(float (&acc)[NCH][ElemTraits<T>::kVec], int r, int gl, unsigned gmask,
+                                           int ch_lo, int ch_hi, int nv, uint4 *stage_rows, T *__restrict__ O0,
+                                           int64_t ldo0, T *__restrict__ O1, int64_t ldo1, int dst_split,
+                                           int accumulate0, const HaloCompress &hc) {
   constexpr int V = ElemTraits<T>::kVec;
-  const int64_t task = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
-  const int gl = threadIdx.x % G;
-  if (task >= (int64_t)rc.count * panels) return;
-  const unsigned lane = threadIdx.x % 32;
-  const unsigned gmask = (G == 32) ? 0xFFFFFFFFu : (((1u << G) - 1u) << (lane & ~(unsigned)(G - 1)));
-  int pos, panel;
-  locate(rc, P, panels, task, pos, panel);
-  const int r = __ldg(rc.rows + pos);
-  const int ch_lo = panel * nv_panel;
-  const int ch_hi = min(nv, ch_lo + nv_panel);
-
-  float acc[NCH][V];
-#pragma unroll
-  for (int i = 0; i < NCH; ++i)
-#pragma unroll
-    for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
-  const int64_t e0 = rp[r];
-  accumulate_range<T, G, NCH, UNR, FULL>(col + e0, val + e0, (int)(rp[r + 1] - e0), gs, ch_lo, ch_hi, gl, gmask, acc);
   if (hc.packed && r >= dst_split) {
     // stage the row in the element type, pick the kept positions, write k values
     typedef typename ElemBits<T>::type E;
@@ -201,6 +190,90 @@ __global__ void __launch_bounds__(256)
       dst[ch] = pack16(acc[i], T());
     }
   }
+}
+
+template <typename T, int G, int NCH, int UNR, bool FULL>
+__global__ void __launch_bounds__(256)
+    spmm_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col, const float *__restrict__ val,
+                RowClass rc, int P, int panels, int nv_panel, GatherSrc gs, T *__restrict__ O0, int64_t ldo0,
+                T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv, HaloCompress hc) {
+  extern __shared__ uint4 stage_rows[];
+  constexpr int V = ElemTraits<T>::kVec;
+  const int64_t task = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+  const int gl = threadIdx.x % G;
+  if (task >= (int64_t)rc.count * panels) return;
+  const unsigned lane = threadIdx.x % 32;
+  const unsigned gmask = (G == 32) ? 0xFFFFFFFFu : (((1u << G) - 1u) << (lane & ~(unsigned)(G - 1)));
+  int pos, panel;
+  locate(rc, P, panels, task, pos, panel);
+  const int r = __ldg(rc.rows + pos);
+  const int ch_lo = panel * nv_panel;
+  const int ch_hi = min(nv, ch_lo + nv_panel);
+
+  float acc[NCH][V];
+#pragma unroll
+  for (int i = 0; i < NCH; ++i)
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
+  const int64_t e0 = rp[r];
+  accumulate_range<T, G, NCH, UNR, FULL>(col + e0, val + e0, (int)(rp[r + 1] - e0), gs, ch_lo, ch_hi, gl, gmask, acc);
+  finish_row<T, G, NCH, FULL>(acc, r, gl, gmask, ch_lo, ch_hi, nv, stage_rows, O0, ldo0, O1, ldo1, dst_split, accumulate0,
+                              hc);
+}
+
+// Short rows (at most 8 entries) from fixed-size records: sources and weights of a row sit at 8 * task, so
+// the gathers start after a single dependent load.
+template <typename T, int G, int NCH, int UNR, bool FULL>
+__global__ void __launch_bounds__(256)
+    spmm_short_kernel(const int32_t *__restrict__ rec_col, const float *__restrict__ rec_val,
+                      const int32_t *__restrict__ rows, int count, GatherSrc gs, T *__restrict__ O0, int64_t ldo0,
+                      T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv, HaloCompress hc) {
+  extern __shared__ uint4 stage_rows[];
+  constexpr int V = ElemTraits<T>::kVec;
+  static_assert(G >= 8, "a record has 8 entries, one per lane");
+  const int task = (blockIdx.x * blockDim.x + threadIdx.x) / G;
+  const int gl = threadIdx.x % G;
+  if (task >= count) return;
+  const unsigned lane = threadIdx.x % 32;
+  const unsigned gmask = (G == 32) ? 0xFFFFFFFFu : (((1u << G) - 1u) << (lane & ~(unsigned)(G - 1)));
+  int myc = -1;
+  float myw = 0.f;
+  if (gl < 8) {
+    myc = __ldg(rec_col + (int64_t)task * 8 + gl);
+    myw = __ldg(rec_val + (int64_t)task * 8 + gl);
+  }
+  const int r = __ldg(rows + task);
+  const int cnt = __popc(__ballot_sync(gmask, myc >= 0) & gmask);
+  const int c_first = __shfl_sync(gmask, myc, 0, G);
+  if (myc < 0) myc = c_first;   // lanes past the row's length: a valid source with weight zero
+  float acc[NCH][V];
+#pragma unroll
+  for (int i = 0; i < NCH; ++i)
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
+  for (int t = 0; t < cnt; t += UNR) {
+    uint4 v[UNR][NCH];
+    float w[UNR];
+#pragma unroll
+    for (int u = 0; u < UNR; ++u) {
+      const int c = __shfl_sync(gmask, myc, t + u, G);
+      w[u] = __shfl_sync(gmask, myw, t + u, G);
+      const bool loc = c < gs.split;
+      const uint4 *src = (loc ? gs.b0 : gs.b1s) + (int64_t)c * (loc ? gs.ld0 : gs.ld1) + gl;
+#pragma unroll
+      for (int i = 0; i < NCH; ++i) v[u][i] = (FULL || gl + i * G < nv) ? __ldg(src + i * G) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < UNR; ++u)
+#pragma unroll
+      for (int i = 0; i < NCH; ++i) {
+        float f[V];
+        unpack16(v[u][i], f, T());
+#pragma unroll
+        for (int j = 0; j < V; ++j) acc[i][j] = fmaf(w[u], f[j], acc[i][j]);
+      }
+  }
+  finish_row<T, G, NCH, FULL>(acc, r, gl, gmask, 0, nv, nv, stage_rows, O0, ldo0, O1, ldo1, dst_split, accumulate0, hc);
 }
 
 // Long rows (hubs of a skewed degree distribution): one CTA per (row, panel), every warp takes a
@@ -332,12 +405,31 @@ int launch_rows(const SpmmArgs &a, const RowClass &rc, cudaStream_t st) {
   return VARCO_OK;
 }
 
+template <typename T, int G, int NCH, int UNR>
+int launch_short(const SpmmArgs &a, cudaStream_t st) {
+  if (a.shorts.count == 0) return VARCO_OK;
+  const int threads = 256;
+  dim3 grid((unsigned)(((int64_t)a.shorts.count * G + threads - 1) / threads));
+  const size_t smem = a.hc.packed ? (size_t)(threads / G) * a.nv * 16 : 0;
+  if (a.nv == G * NCH)
+    spmm_short_kernel<T, G, NCH, UNR, true><<<grid, threads, smem, st>>>(
+        a.short_col, a.short_val, a.shorts.rows, a.shorts.count, gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1,
+        a.dst_split, a.accumulate0, a.nv, a.hc);
+  else
+    spmm_short_kernel<T, G, NCH, UNR, false><<<grid, threads, smem, st>>>(
+        a.short_col, a.short_val, a.shorts.rows, a.shorts.count, gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1,
+        a.dst_split, a.accumulate0, a.nv, a.hc);
+  VARCO_KERNEL_LAUNCHED();
+  return VARCO_OK;
+}
+
 // G/NCH: lanes per row and 16-byte chunks per lane for ordinary rows; GS/NCHS: the same for rows of
 // at most a handful of entries, where narrower groups keep more rows in flight per warp.
 template <typename T, int G, int NCH, int UNR, int GS, int NCHS, int UNRS>
 int launch(const SpmmArgs &a, cudaStream_t st) {
   if (int rc = launch_hubs<T, NCH, UNR>(a, st)) return rc;
   if (int rc = launch_rows<T, G, NCH, UNR>(a, a.normal, st)) return rc;
+  if (a.panels == 1 && a.short_col) return launch_short<T, (GS < 8 ? 8 : GS), (GS < 8 ? (NCHS * GS + 7) / 8 : NCHS), VARCO_SHORT_UNR>(a, st);
   return launch_rows<T, GS, NCHS, UNRS>(a, a.shorts, st);
 }
 
@@ -604,6 +696,8 @@ int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, cons
   a.nv = nv;
   a.panels = 1;
   a.nv_panel = nv;
+  a.short_col = pl->d.short_f_col;
+  a.short_val = pl->d.short_f_val;
   return dt == VARCO_F32 ? dispatch<float>(a, st) : dispatch<__nv_bfloat16>(a, st);
 }
 
@@ -675,6 +769,8 @@ int varco_launch_spmm_bwd(const varco_plan *pl, const void *dAgg, int64_t ldd, i
   a.nv = nv;
   a.panels = 1;
   a.nv_panel = nv;
+  a.short_col = pl->d.short_t_col;
+  a.short_val = pl->d.short_t_val;
   if (packed) a.hc = HaloCompress{packed, kstride, k, F, vperm::half_bits(F), vperm::layer_key(key), pl->d.slot_gid};
   return dt == VARCO_F32 ? dispatch<float>(a, st) : dispatch<__nv_bfloat16>(a, st);
 }

@@ -37,6 +37,9 @@ struct varco_dev_image {
   const int32_t *hub_t = nullptr;
   const int32_t *short_f = nullptr;
   const int32_t *short_t = nullptr;
+  // 8-entry records of the short rows (sources, weights), in class-list order
+  const int32_t *short_f_col = nullptr, *short_t_col = nullptr;
+  const float *short_f_val = nullptr, *short_t_val = nullptr;
   // [P + 1] first position of every partition in the class lists above
   const int32_t *order_f_start = nullptr, *order_t_start = nullptr, *hub_f_start = nullptr, *hub_t_start = nullptr,
                 *short_f_start = nullptr, *short_t_start = nullptr;
@@ -54,7 +57,8 @@ struct varco_plan {
   std::vector<int32_t> order_f, order_t, hub_f, hub_t, short_f, short_t, nloc;
   std::vector<int32_t> order_f_start, order_t_start, hub_f_start, hub_t_start, short_f_start, short_t_start;
   std::vector<int64_t> rp, rpT;
-  std::vector<float> val, valT;
+  std::vector<float> val, valT, short_f_val, short_t_val;
+  std::vector<int32_t> short_f_col, short_t_col;
   // device image
   bool uploaded = false;
   varco_dev_image d;
