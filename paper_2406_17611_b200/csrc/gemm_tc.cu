@@ -34,7 +34,10 @@ constexpr int kBlockM = 128;     // UMMA M
 constexpr int kBlockK = 64;      // bf16 elements per 128-byte swizzle span
 constexpr int kUmmaK = 16;
 constexpr uint32_t kTmemCols = 512;
-constexpr int kThreads = 192;    // warps 0-3 epilogue, 4 TMA, 5 MMA
+constexpr int kThreads = 320;    // warps 0-7 epilogue (two per TMEM lane quarter), 8 TMA, 9 MMA
+constexpr int kEpiWarps = 8;
+constexpr int kTmaWarp = 8, kMmaWarp = 9;
+constexpr int kThreadsDw = 192;  // dW kernel: warps 0-3 epilogue, 4 TMA, 5 MMA
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr long long kSpinClocks = 2000000000ll;   // about one second of SM clocks
 
@@ -143,6 +146,7 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn_major, 
 struct RowsParams {
   CUtensorMap tmA[2];   // activations, box {64, 128}
   CUtensorMap tmB;      // packed weights [n_tiles * N_tile rows][(kb0 + kb1) * 64], box {64, N_tile}
+  CUtensorMap tmOut[4]; // outputs of the n tiles: [M x valid columns], box {64, 32}, for the epilogue's stores
   int kblocks[2];
   int num_a;
   int M, m_tiles, n_tiles, N_tile;
@@ -170,7 +174,8 @@ __global__ void __launch_bounds__(kThreads, 1) rows_kernel(const __grid_constant
   const uint32_t b_stride = 256 * kBlockK * 2;
   uint8_t *sA = base;
   uint8_t *sB = base + kStagesRows * a_bytes;
-  RowsSmem *sh = reinterpret_cast<RowsSmem *>(sB + kStagesRows * b_stride);
+  uint8_t *stage_base = sB + kStagesRows * b_stride;   // 8 x 4 KB epilogue tiles (1024-byte aligned)
+  RowsSmem *sh = reinterpret_cast<RowsSmem *>(stage_base + 8 * 4096);
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   volatile int *abort_flag = &sh->abort_flag;
 
@@ -181,14 +186,14 @@ __global__ void __launch_bounds__(kThreads, 1) rows_kernel(const __grid_constant
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(&sh->tfull[a], 1);
-      mbar_init(&sh->tempty[a], 4);
+      mbar_init(&sh->tempty[a], kEpiWarps);
     }
     sh->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   for (int i = threadIdx.x; i < 256; i += kThreads)
     sh->bias[i] = (p.bias && i < p.ncols[0]) ? p.bias[i] : 0.f;
-  if (warp == 5) tmem_alloc(&sh->tmem_base, kTmemCols);
+  if (warp == kMmaWarp) tmem_alloc(&sh->tmem_base, kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -196,7 +201,7 @@ __global__ void __launch_bounds__(kThreads, 1) rows_kernel(const __grid_constant
   const int total_work = p.m_tiles * p.n_tiles;
   const int ksteps = p.kblocks[0] + (p.num_a > 1 ? p.kblocks[1] : 0);
 
-  if (warp == 4) {
+  if (warp == kTmaWarp) {
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
@@ -226,7 +231,7 @@ __global__ void __launch_bounds__(kThreads, 1) rows_kernel(const __grid_constant
             if (mbar_try_wait(&sh->full[s], 0) || mbar_try_wait(&sh->full[s], 1)) break;
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kMmaWarp) {
     if (lane == 0) {
       const uint32_t idesc = instr_desc(kBlockM, p.N_tile, 0, 0);
       int stage = 0;
@@ -263,7 +268,8 @@ __global__ void __launch_bounds__(kThreads, 1) rows_kernel(const __grid_constant
       }
     }
   } else {
-    // epilogue warps 0..3: warp w owns TMEM lanes [32 w, 32 w + 32) = tile rows
+    // epilogue warps: warp w reads TMEM lanes [32 (w % 4), + 32) = tile rows and takes every second
+    // 64-column slab, starting with slab w / 4
     int local = 0;
     for (int w = blockIdx.x; w < total_work; w += gridDim.x, ++local) {
       const int mt = w / p.n_tiles, nt = w % p.n_tiles;
@@ -271,38 +277,54 @@ __global__ void __launch_bounds__(kThreads, 1) rows_kernel(const __grid_constant
       const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
       if (!mbar_wait(&sh->tfull[acc], acc_phase, abort_flag, p.err, 4)) break;
       tc_fence_after();
-      const int row = mt * kBlockM + warp * 32 + lane;
-      const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)acc * 256u;
-      __nv_bfloat16 *orow = p.out[nt] + (int64_t)row * p.ldo[nt] + p.col0[nt];
+      const int quarter = warp & 3;
+      const int row0 = mt * kBlockM + quarter * 32;          // first tile row of this warp
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * 256u;
       const int ncols = p.ncols[nt];
-      const int room = (int)(p.ldo[nt] - p.col0[nt]);
-      for (int c0 = 0; c0 < p.N_tile; c0 += 16) {
-        uint32_t r[16];
-        tmem_ld16(taddr + (uint32_t)c0, r);
+      // A thread holds one ROW of the accumulator, so storing from registers would touch 32 different lines
+      // per instruction.  Instead every 64-column slab goes to a 128-byte-swizzled shared-memory tile
+      // (32 rows x 128 B per warp) and leaves through one TMA store, which also clips the ragged edges.
+      uint4 *stg = reinterpret_cast<uint4 *>(stage_base + (size_t)warp * 4096);   // one staging tile per warp
+      for (int c64 = (warp >> 2) * 64; c64 < p.N_tile && c64 < ncols; c64 += 128) {
+        uint32_t r[4][16];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          if (c64 + q * 16 < p.N_tile) tmem_ld16(taddr + (uint32_t)(c64 + q * 16), r[q]);
         tmem_ld_wait();
-        if (row < p.M && c0 < ncols) {
+        const bool plain = !p.bias && !p.relu && c64 + 64 <= ncols && c64 + 64 <= p.N_tile;
+        // the previous store of this warp must have finished reading the tile
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        __syncwarp();
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int c0 = c64 + q * 16;
           float f[16];
+          if (plain) {   // no bias, no activation, slab fully inside the valid columns: convert only
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            float v = __uint_as_float(r[j]);
-            if (p.bias) v += sh->bias[c0 + j];
-            if (p.relu) v = fmaxf(v, 0.f);
-            f[j] = (c0 + j < ncols) ? v : 0.f;
-          }
+            for (int j = 0; j < 16; ++j) f[j] = __uint_as_float(r[q][j]);
+          } else {
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            const int c = c0 + half * 8;
-            if (c + 8 <= room) {
-              uint4 pk = make_uint4(pack_bf16x2(f[half * 8 + 0], f[half * 8 + 1]),
-                                    pack_bf16x2(f[half * 8 + 2], f[half * 8 + 3]),
-                                    pack_bf16x2(f[half * 8 + 4], f[half * 8 + 5]),
-                                    pack_bf16x2(f[half * 8 + 6], f[half * 8 + 7]));
-              *reinterpret_cast<uint4 *>(orow + c) = pk;
-            } else {
-              for (int j = 0; j < 8; ++j)
-                if (c + j < ncols) orow[c + j] = __float2bfloat16_rn(f[half * 8 + j]);
+            for (int j = 0; j < 16; ++j) {
+              float v = c0 < p.N_tile ? __uint_as_float(r[q][j]) : 0.f;
+              if (p.bias) v += sh->bias[(c0 + j) & 255];
+              if (p.relu) v = fmaxf(v, 0.f);
+              f[j] = (c0 + j < ncols) ? v : 0.f;
             }
           }
+          // 16-byte chunk j of row `lane` sits at chunk position j ^ (lane & 7)
+          stg[lane * 8 + ((q * 2) ^ (lane & 7))] = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]),
+                                                              pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+          stg[lane * 8 + ((q * 2 + 1) ^ (lane & 7))] = make_uint4(pack_bf16x2(f[8], f[9]), pack_bf16x2(f[10], f[11]),
+                                                                  pack_bf16x2(f[12], f[13]), pack_bf16x2(f[14], f[15]));
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
+                           reinterpret_cast<uint64_t>(&p.tmOut[nt])),
+                       "r"(p.col0[nt] + c64), "r"(row0), "r"(smem_u32(stg))
+                       : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
       }
       tc_fence_before();
@@ -310,10 +332,11 @@ __global__ void __launch_bounds__(kThreads, 1) rows_kernel(const __grid_constant
       if (lane == 0) mbar_arrive(&sh->tempty[acc]);
     }
   }
+  if (warp < kEpiWarps && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if (warp == 5) tmem_dealloc(tmem_base, kTmemCols);
+  if (warp == kMmaWarp) tmem_dealloc(tmem_base, kTmemCols);
 }
 
 // ------------------------------------------------------------------------------------------ kernel 2
@@ -337,7 +360,7 @@ struct DwSmem {
   int abort_flag;
 };
 
-__global__ void __launch_bounds__(kThreads, 1) dw_kernel(const __grid_constant__ DwParams p) {
+__global__ void __launch_bounds__(kThreadsDw, 1) dw_kernel(const __grid_constant__ DwParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   constexpr uint32_t box_bytes = 64 * 64 * 2;             // 8 KB: 64 nodes x 128 B
@@ -478,6 +501,7 @@ __global__ void dw_reduce_kernel(const float *__restrict__ partial, int splits, 
 // Weight repack for kernel 1.
 //  mode 0 (forward):  B[o][koff_a + c] = W_a[c][o]      rows = outputs, K = [X block | Agg block], zero padded
 //  mode 1 (backward): B[t * N_tile + j][c] = W_t[j][c]  rows = input features of operand t, K = outputs
+//  mode 2 (backward, concatenated K): B[j][a * koff1 + c] = W_a[j][c]  rows = input features, K = [op 0 | op 1]
 __global__ void pack_weights_kernel(const __nv_bfloat16 *__restrict__ W0, const __nv_bfloat16 *__restrict__ W1,
                                     int F_in, int F_out, int mode, int rows, int kcols, int koff1, int N_tile,
                                     int tiles_per_op, __nv_bfloat16 *__restrict__ B) {
@@ -490,6 +514,11 @@ __global__ void pack_weights_kernel(const __nv_bfloat16 *__restrict__ W0, const 
     const int cc = a ? c - koff1 : c;
     const __nv_bfloat16 *W = a ? W1 : W0;
     if (r < F_out && cc < F_in) v = W[(int64_t)cc * F_out + r];
+  } else if (mode == 2) {
+    const int a = (W1 && c >= koff1) ? 1 : 0;
+    const int cc = a ? c - koff1 : c;
+    const __nv_bfloat16 *W = a ? W1 : W0;
+    if (r < F_in && cc < F_out) v = W[(int64_t)r * F_out + cc];
   } else {
     const int tile = r / N_tile, j = r % N_tile;
     const int op = tile / tiles_per_op;
@@ -546,7 +575,7 @@ int sm_count() {
 }
 
 constexpr size_t rows_smem_bytes() {
-  return 1024 + kStagesRows * (size_t)(kBlockM * kBlockK * 2 + 256 * kBlockK * 2) + sizeof(RowsSmem) + 64;
+  return 1024 + kStagesRows * (size_t)(kBlockM * kBlockK * 2 + 256 * kBlockK * 2) + 8 * 4096 + sizeof(RowsSmem) + 64;
 }
 constexpr size_t dw_smem_bytes() { return 1024 + kStagesDw * (size_t)(8 * 64 * 64 * 2) + sizeof(DwSmem) + 64; }
 
@@ -589,6 +618,13 @@ static int configure_once() {
   return rc;
 }
 
+// tensor maps of the epilogue's stores: tile t writes columns [col0, col0 + ncols) of its destination
+static int make_out_maps(RowsParams &p) {
+  for (int t = 0; t < p.n_tiles; ++t)
+    if (make_map(&p.tmOut[t], p.out[t], p.M, p.col0[t] + p.ncols[t], p.ldo[t], 32)) return VARCO_CUDA;
+  return VARCO_OK;
+}
+
 // Y[n x F_out] = act([X | Agg] [Ws ; Wn] + bias); Ws == nullptr: Y = act(Agg Wn + bias)
 int varco_tc_gemm_fwd(int n, int F_in, int F_out, const void *X, int64_t ldx, const void *Agg, int64_t lda,
                       const void *Ws, const void *Wn, const float *bias, int relu, void *Y, int64_t ldy,
@@ -629,6 +665,7 @@ int varco_tc_gemm_fwd(int n, int F_in, int F_out, const void *X, int64_t ldx, co
   p.relu = relu;
   p.err = err;
   const int grid = p.m_tiles < sm_count() ? p.m_tiles : sm_count();
+  if (make_out_maps(p)) return VARCO_CUDA;
   rows_kernel<<<grid, kThreads, rows_smem_bytes(), st>>>(p);
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
@@ -678,6 +715,55 @@ int varco_tc_gemm_dx(int n, int F_in, int F_out, const void *dZ, int64_t lddz, c
   p.err = err;
   const int work = p.m_tiles * p.n_tiles;
   const int grid = work < sm_count() ? work : sm_count();
+  if (make_out_maps(p)) return VARCO_CUDA;
+  rows_kernel<<<grid, kThreads, rows_smem_bytes(), st>>>(p);
+  VARCO_KERNEL_LAUNCHED();
+  return VARCO_OK;
+}
+
+// out[m x F_in] = A0 W0^T (+ A1 W1^T), A_a being [m x F_out] and W_a [F_in x F_out]: the backward products
+// with the K range concatenated over the two operands.
+int varco_tc_gemm_cat_t(int m, int F_in, int F_out, const void *A0, int64_t lda0, const void *A1, int64_t lda1,
+                        const void *W0, const void *W1, void *out, int64_t ldo, void *scratch, int *err,
+                        cudaStream_t st) {
+  if (configure_once() != VARCO_OK) return VARCO_CUDA;
+  TcScratch sc = carve(scratch, F_in, F_out);
+  RowsParams p;
+  memset(&p, 0, sizeof(p));
+  const int tiles = ceil_div(F_in, 256);
+  const int N_tile = ceil_div(ceil_div(F_in, tiles), 16) * 16;
+  if (tiles > 4) return VARCO_UNSUPPORTED;
+  const int kb = ceil_div(F_out, 64);
+  p.num_a = A1 ? 2 : 1;
+  p.kblocks[0] = kb;
+  p.kblocks[1] = A1 ? kb : 0;
+  const int kcols = (p.kblocks[0] + p.kblocks[1]) * 64;
+  const int rows = tiles * N_tile;
+  if (make_map(&p.tmA[0], A0, m, F_out, lda0, 128)) return VARCO_CUDA;
+  if (A1 && make_map(&p.tmA[1], A1, m, F_out, lda1, 128)) return VARCO_CUDA;
+  if (make_map(&p.tmB, sc.packed, rows, kcols, kcols, N_tile)) return VARCO_CUDA;
+  {
+    const int64_t total = (int64_t)rows * kcols;
+    pack_weights_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
+        (const __nv_bfloat16 *)W0, (const __nv_bfloat16 *)(A1 ? W1 : nullptr), F_in, F_out, 2, rows, kcols, kb * 64,
+        N_tile, 1, sc.packed);
+    VARCO_KERNEL_LAUNCHED();
+  }
+  p.M = m;
+  p.m_tiles = ceil_div(m, kBlockM);
+  p.n_tiles = tiles;
+  p.N_tile = N_tile;
+  for (int t = 0; t < tiles; ++t) {
+    p.out[t] = (__nv_bfloat16 *)out;
+    p.ldo[t] = ldo;
+    p.col0[t] = t * N_tile;
+    const int nc = F_in - t * N_tile;
+    p.ncols[t] = nc > N_tile ? N_tile : nc;
+  }
+  p.err = err;
+  const int64_t work = (int64_t)p.m_tiles * p.n_tiles;
+  const int grid = work < sm_count() ? (int)work : sm_count();
+  if (make_out_maps(p)) return VARCO_CUDA;
   rows_kernel<<<grid, kThreads, rows_smem_bytes(), st>>>(p);
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
@@ -716,7 +802,7 @@ int varco_tc_gemm_dw(int n, int F_in, int F_out, const void *X, int64_t ldx, con
   p.partial = sc.partial;
   p.err = err;
   dim3 grid(splits, groups);
-  dw_kernel<<<grid, kThreads, dw_smem_bytes(), st>>>(p);
+  dw_kernel<<<grid, kThreadsDw, dw_smem_bytes(), st>>>(p);
   VARCO_KERNEL_LAUNCHED();
   const int64_t total = (int64_t)num_ops * F_in * F_out;
   dw_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(sc.partial, splits, p.N_pad, F_in, F_out,

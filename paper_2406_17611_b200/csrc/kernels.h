@@ -57,6 +57,9 @@ int varco_tc_gemm_fwd(int n, int F_in, int F_out, const void *X, int64_t ldx, co
                       void *scratch, int *err, cudaStream_t st);
 int varco_tc_gemm_dx(int n, int F_in, int F_out, const void *dZ, int64_t lddz, const void *Ws, const void *Wn,
                      void *dXs, int64_t ldxs, void *dAgg, int64_t ldagg, void *scratch, int *err, cudaStream_t st);
+int varco_tc_gemm_cat_t(int m, int F_in, int F_out, const void *A0, int64_t lda0, const void *A1, int64_t lda1,
+                        const void *W0, const void *W1, void *out, int64_t ldo, void *scratch, int *err,
+                        cudaStream_t st);
 int varco_tc_gemm_dw(int n, int F_in, int F_out, const void *X, int64_t ldx, const void *Agg, int64_t lda,
                      const void *dZ, int64_t lddz, float *dWs, float *dWn, void *scratch, int *err, cudaStream_t st);
 

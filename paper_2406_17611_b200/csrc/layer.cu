@@ -211,6 +211,34 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
     if (rc == VARCO_OK && dbias) rc = varco_colsum(n, F_out, dt, dZ, lddz, dbias, scratch, st);
   }
   if (rc != VARCO_OK) return rc;
+  // Narrow backward (full communication, F_out well below F_in, tensor-core path): aggregation and the
+  // weight product commute, so the transposed aggregation runs on the F_out-wide dZ instead of the F_in-wide
+  // dZ W_neigh^T, and the product with W_neigh^T is applied afterwards to the local sums and to the slot sums.
+  const bool narrow = tc && k == F_in && 2 * L.ld_out <= F_in;
+  if (narrow) {
+    void *Gl = dAgg;      // [n x ld_out] local sums of dZ
+    void *Gh = packed;    // [H x ld_out] slot sums of dZ
+    {
+      StageTimer t(plan, VARCO_STAGE_SPMM_T, stream);
+      rc = varco_launch_spmm_bwd(plan, dZ, lddz, F_out, dt, Gl, L.ld_out, 0, Gh, L.ld_out, nullptr, 0, 0, key, st);
+    }
+    if (rc != VARCO_OK) return rc;
+    {
+      StageTimer t(plan, VARCO_STAGE_GEMM_DX, stream);
+      if (sage)
+        rc = varco_tc_gemm_cat_t(n, F_in, F_out, dZ, lddz, Gl, L.ld_out, W_self, W_neigh, dX, desc->ld_in, scratch,
+                                 status, st);
+      else
+        rc = varco_tc_gemm_cat_t(n, F_in, F_out, Gl, L.ld_out, nullptr, 0, W_neigh, nullptr, dX, desc->ld_in, scratch,
+                                 status, st);
+      if (rc == VARCO_OK && plan->H > 0)
+        rc = varco_tc_gemm_cat_t((int)plan->H, F_in, F_out, Gh, L.ld_out, nullptr, 0, W_neigh, nullptr, Ghalo, L.ld_in,
+                                 scratch, status, st);
+    }
+    if (rc != VARCO_OK) return rc;
+    StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
+    return varco_launch_add_dense_rows(plan, Ghalo, L.ld_in, F_in, dt, dX, desc->ld_in, st);
+  }
   {
     StageTimer t(plan, VARCO_STAGE_GEMM_DX, stream);
     if (tc) {
