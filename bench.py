@@ -185,6 +185,22 @@ class DeviceModel:
         return h2d, d2h
 
 
+def measured_traffic(args, stage):
+    """DRAM bytes per epoch of one stage from the committed ncu capture, or None when the capture does not
+    belong to this workload / ratio or was taken from other kernel sources."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic_c3_ratio1.json")
+    if args.workload != "c3" or args.scale != 1.0 or parse_ratio(args.ratio) != (1, 1) or args.parts:
+        return None
+    try:
+        from paper_2406_17611_b200.ncu_summary import source_digest
+        d = json.load(open(path))
+        if d.get("source_sha1") != source_digest():
+            return None
+        return d["dram_bytes_per_epoch"].get(stage)
+    except (OSError, ValueError, KeyError):
+        return None
+
+
 def stage_work(wl, plan, ratio_k):
     """Algorithmic bytes / flops of every stage for ONE epoch (all layers), as the design doc derives."""
     n, nnz, H = wl.n, plan.nnz, plan.H_total
@@ -399,6 +415,10 @@ def run_ours(args):
     else:
         roof = {"kernel": dom, "bound": "hbm", "achieved": d["gbs"], "peak": pk["hbm_gbs"], "unit": "GB/s",
                 "frac": d["gbs"] / pk["hbm_gbs"], "traffic": None, "peak_source": pk["source"]}
+
+    roof["traffic"] = measured_traffic(args, dom)
+    roof["algorithmic"] = work.get(dom)
+    roof["per"] = "epoch (all launches of the stage)"
 
     # epoch time versus rate
     sweep = {}

@@ -247,13 +247,15 @@ int varco_workspace_status(const void *workspace, void *stream, int *device_stat
  */
 enum {
   VARCO_STAGE_COMPRESS = 0,      /* halo gather + compress (forward)            */
-  VARCO_STAGE_DECOMPRESS = 1,    /* decompress + scatter into halo slots        */
+  VARCO_STAGE_DECOMPRESS = 1,    /* decompress into halo slots (dense rows, or
+                                    (value, position) pairs when k <= F/8)      */
   VARCO_STAGE_SPMM = 2,          /* aggregation over local + halo rows          */
   VARCO_STAGE_GEMM_FWD = 3,      /* feature transform, bias, activation         */
   VARCO_STAGE_GEMM_DX = 4,       /* dZ W^T                                       */
   VARCO_STAGE_GEMM_DW = 5,       /* [X | Agg]^T dZ and dbias                     */
   VARCO_STAGE_SPMM_T = 6,        /* transposed aggregation (to rows and slots)   */
-  VARCO_STAGE_COMPRESS_BWD = 7,  /* compress halo-slot gradients                 */
+  VARCO_STAGE_COMPRESS_BWD = 7,  /* unused: the gradient compression runs in the
+                                    epilogue of the transposed aggregation (stage 6) */
   VARCO_STAGE_SCATTER_ADD = 8,   /* decompress + ordered add into owner rows     */
   VARCO_STAGE_AUX = 9,           /* small helpers: masks, casts, weight repacks  */
   VARCO_STAGE_COUNT = 10

@@ -241,6 +241,19 @@ __global__ void __launch_bounds__(256) add_dense_rows_kernel(const T *__restrict
     float acc[V];
     unpack16(row4[v], acc, T());
     int s = s0;
+    for (; s + 3 < s1; s += 4) {   // four slot rows in flight, added in ascending slot order
+      uint4 q[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        q[u] = __ldg(reinterpret_cast<const uint4 *>(Gh + (int64_t)brow_slot[s + u] * ldg) + v);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        float f[V];
+        unpack16(q[u], f, T());
+#pragma unroll
+        for (int i = 0; i < V; ++i) acc[i] += f[i];
+      }
+    }
     for (; s + 1 < s1; s += 2) {
       const uint4 a = __ldg(reinterpret_cast<const uint4 *>(Gh + (int64_t)brow_slot[s] * ldg) + v);
       const uint4 c = __ldg(reinterpret_cast<const uint4 *>(Gh + (int64_t)brow_slot[s + 1] * ldg) + v);

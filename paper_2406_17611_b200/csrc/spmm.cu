@@ -278,7 +278,7 @@ __global__ void __launch_bounds__(256)
 
 // Long rows (hubs of a skewed degree distribution): one CTA per (row, panel), every warp takes a
 // contiguous share of the entries, partial sums meet in shared memory and are added in warp order.
-template <typename T, int NCH, int UNR, bool FULL>
+template <typename T, int G, int NCH, int UNR, bool FULL>
 __global__ void __launch_bounds__(256)
     spmm_hub_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col, const float *__restrict__ val,
                     RowClass rc, int P, int panels, int nv_panel, GatherSrc gs, T *__restrict__ O0, int64_t ldo0,
@@ -293,8 +293,15 @@ __global__ void __launch_bounds__(256)
   const int ch_lo = panel * nv_panel;
   const int ch_hi = min(nv, ch_lo + nv_panel);
   const int64_t e0 = rp[r], e1 = rp[r + 1];
-  const int64_t per = ((e1 - e0 + nwarps - 1) / nwarps + 31) / 32 * 32;
-  const int64_t b0 = e0 + warp * per < e1 ? e0 + warp * per : e1;
+  // the entries are shared out over the warps, and inside a warp over its 32 / G lane groups (narrow rows
+  // need fewer than 32 lanes per gathered row); the groups' sums meet by a fixed shuffle tree
+  constexpr int kGroups = 32 / G;
+  const int gl = lane % G, gi = lane / G;
+  const unsigned gmask = (G == 32) ? 0xFFFFFFFFu : (((1u << G) - 1u) << (lane & ~(unsigned)(G - 1)));
+  const int64_t shares = (int64_t)nwarps * kGroups;
+  const int64_t per = ((e1 - e0 + shares - 1) / shares + G - 1) / G * G;
+  const int64_t mine = (int64_t)warp * kGroups + gi;
+  const int64_t b0 = e0 + mine * per < e1 ? e0 + mine * per : e1;
   const int64_t b1 = b0 + per < e1 ? b0 + per : e1;
   float acc[NCH][V];
 #pragma unroll
@@ -302,13 +309,18 @@ __global__ void __launch_bounds__(256)
 #pragma unroll
     for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
   if (b1 > b0)
-    accumulate_range<T, 32, NCH, UNR, FULL>(col + b0, val + b0, (int)(b1 - b0), gs, ch_lo, ch_hi, lane, 0xFFFFFFFFu,
-                                            acc);
+    accumulate_range<T, G, NCH, UNR, FULL>(col + b0, val + b0, (int)(b1 - b0), gs, ch_lo, ch_hi, gl, gmask, acc);
+#pragma unroll
+  for (int off = G; off < 32; off <<= 1)
+#pragma unroll
+    for (int i = 0; i < NCH; ++i)
+#pragma unroll
+      for (int j = 0; j < V; ++j) acc[i][j] += __shfl_xor_sync(0xFFFFFFFFu, acc[i][j], off);
   const int row_floats = nv_panel * V;
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
-    const int c = lane + i * 32;
-    if (c < nv_panel)
+    const int c = gl + i * G;
+    if (gi == 0 && c < nv_panel)
 #pragma unroll
       for (int j = 0; j < V; ++j) hub_part[(size_t)warp * row_floats + c * V + j] = acc[i][j];
   }
@@ -366,7 +378,7 @@ GatherSrc gather_src(const SpmmArgs &a) {
   return gs;
 }
 
-template <typename T, int NCH, int UNR>
+template <typename T, int G, int NCH, int UNR>
 int launch_hubs(const SpmmArgs &a, cudaStream_t st) {
   if (a.hubs.count == 0) return VARCO_OK;
   constexpr int V = ElemTraits<T>::kVec;
@@ -374,12 +386,12 @@ int launch_hubs(const SpmmArgs &a, cudaStream_t st) {
   int warps = 8;
   while (warps > 1 && warps * row_bytes > 48 * 1024) warps /= 2;
   const dim3 grid((unsigned)(a.hubs.count * a.panels));
-  if (a.panels == 1 && a.nv == 32 * NCH)
-    spmm_hub_kernel<T, NCH, UNR, true><<<grid, warps * 32, warps * row_bytes, st>>>(
+  if (a.panels == 1 && a.nv == G * NCH)
+    spmm_hub_kernel<T, G, NCH, UNR, true><<<grid, warps * 32, warps * row_bytes, st>>>(
         a.rp, a.col, a.val, a.hubs, a.P, a.panels, a.nv_panel, gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1,
         a.dst_split, a.accumulate0, a.nv, a.hc);
   else
-    spmm_hub_kernel<T, NCH, UNR, false><<<grid, warps * 32, warps * row_bytes, st>>>(
+    spmm_hub_kernel<T, G, NCH, UNR, false><<<grid, warps * 32, warps * row_bytes, st>>>(
         a.rp, a.col, a.val, a.hubs, a.P, a.panels, a.nv_panel, gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1,
         a.dst_split, a.accumulate0, a.nv, a.hc);
   VARCO_KERNEL_LAUNCHED();
@@ -427,7 +439,7 @@ int launch_short(const SpmmArgs &a, cudaStream_t st) {
 // at most a handful of entries, where narrower groups keep more rows in flight per warp.
 template <typename T, int G, int NCH, int UNR, int GS, int NCHS, int UNRS>
 int launch(const SpmmArgs &a, cudaStream_t st) {
-  if (int rc = launch_hubs<T, NCH, UNR>(a, st)) return rc;
+  if (int rc = launch_hubs<T, (G < 8 ? 8 : G), (G < 8 ? 1 : NCH), UNR>(a, st)) return rc;
   if (int rc = launch_rows<T, G, NCH, UNR>(a, a.normal, st)) return rc;
   if (a.panels == 1 && a.short_col) return launch_short<T, (GS < 8 ? 8 : GS), (GS < 8 ? (NCHS * GS + 7) / 8 : NCHS), VARCO_SHORT_UNR>(a, st);
   return launch_rows<T, GS, NCHS, UNRS>(a, a.shorts, st);

@@ -202,7 +202,7 @@ def test_hub_rows(orc, bf16, F_in, F_out):
     perm = plan.perm()
     ws = plan.workspace(F_in, F_out, vb.BF16 if bf16 else vb.F32)
     Xd = to_device_rows(X, perm, dt)
-    for ratio in [(1, 1), (4, 1)]:
+    for ratio in [(1, 1), (4, 1), (32, 1)]:   # full, dense-compressed, sparse-halo paths
         key = (9, 1, 0)
         Y, Agg, _ = vb.varco_layer_fwd(plan, Xd, dev_weights(Ws, dt), dev_weights(Wn, dt),
                                        dev_weights(b, torch.float32), True, ratio, key, ws, F_in=F_in)
