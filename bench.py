@@ -151,8 +151,7 @@ class DeviceModel:
     def _ld(self, f):
         return (f + self.vec - 1) // self.vec * self.vec
 
-    def epoch(self, ratio, epoch_idx):
-        """All layers forward then backward.  Returns the halo bytes put on the wire."""
+    def _forward(self, ratio, epoch_idx):
         vb, wl = self.vb, self.wl
         total = 0
         for l in range(self.L):
@@ -161,6 +160,11 @@ class DeviceModel:
                                           (wl.seed, epoch_idx, l), self.ws, F_in=wl.widths[l], Y=self.acts[l + 1],
                                           Agg=self.aggs[l])
             total += hb
+        return total
+
+    def _backward(self, ratio, epoch_idx):
+        vb, wl = self.vb, self.wl
+        total = 0
         for l in reversed(range(self.L)):
             w = self.W[l]
             r = vb.varco_layer_bwd(self.plan, self.acts[l], self.acts[l + 1], self.aggs[l], w["Ws"], w["Wn"],
@@ -170,12 +174,32 @@ class DeviceModel:
             total += r[4]
         return total
 
+    def epoch(self, ratio, epoch_idx):
+        """All layers forward then backward.  Returns the halo bytes put on the wire."""
+        return self._forward(ratio, epoch_idx) + self._backward(ratio, epoch_idx)
+
     def epoch_e2e(self, ratio, epoch_idx):
-        """The same epoch fed from pinned host memory, results read back to the host."""
+        """The same epoch fed from pinned host memory, results read back to the host.  X_0 must arrive before
+        the forward pass starts; the upstream gradient is only needed by the backward pass and the logits are
+        final after the forward pass, so those two copies run on a second stream beside the kernels."""
+        torch = self.torch
+        main = torch.cuda.current_stream()
+        if not hasattr(self, "_copy_stream"):
+            self._copy_stream = torch.cuda.Stream()
+        side = self._copy_stream
+        side.wait_stream(main)                      # the previous step has released the buffers
         self.acts[0].copy_(self.X0_host, non_blocking=True)
-        self.grads[self.L].copy_(self.dY_host, non_blocking=True)
-        self.epoch(ratio, epoch_idx)
-        self.Y_host.copy_(self.acts[self.L], non_blocking=True)
+        with torch.cuda.stream(side):
+            self.grads[self.L].copy_(self.dY_host, non_blocking=True)
+            dY_ready = side.record_event()
+        total = self._forward(ratio, epoch_idx)
+        fwd_done = main.record_event()
+        with torch.cuda.stream(side):
+            side.wait_event(fwd_done)
+            self.Y_host.copy_(self.acts[self.L], non_blocking=True)
+        main.wait_event(dY_ready)
+        total += self._backward(ratio, epoch_idx)
+        main.wait_stream(side)
         host = [w["dWn"].cpu() for w in self.W]
         return host
 

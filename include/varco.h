@@ -98,6 +98,10 @@ int varco_partition_info(const varco_plan_t *plan, int64_t *n, int64_t *nnz, int
                          int64_t *H_total, int64_t *cross_entries, int64_t *self_entries);
 /* Number of distinct rows that are a halo row of at least one other partition. */
 int varco_partition_boundary_rows(const varco_plan_t *plan, int64_t *count);
+/* Tuning knob (no counterpart in the paper), off by default.  With bytes > 0 the forward aggregation splits the
+ * feature row into panels so that the rows one partition gathers from (its own plus its halo slots) fit in
+ * `bytes` of L2.  On B200 this did not pay on the measured workloads; results are unchanged either way. */
+int varco_partition_set_l2_budget(varco_plan_t *plan, int64_t bytes);
 /* PxP[p * P + q] = |halo(p->q)| (host array of P*P entries). */
 int varco_partition_counts(const varco_plan_t *plan, int64_t *PxP);
 /* Original ids of halo(p->q), ascending; the pointer stays valid until the plan is destroyed. */

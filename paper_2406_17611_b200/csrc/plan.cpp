@@ -104,6 +104,9 @@ int build(varco_plan *pl, int64_t n, const int64_t *rp0, const int32_t *col0, co
   std::vector<int64_t> slot_base(P + 1, 0);
   for (int q = 0; q < P; ++q) slot_base[q + 1] = slot_base[q] + (int64_t)recv[q].size();
   pl->H = slot_base[P];
+  for (int q = 0; q < P; ++q)
+    pl->max_part_sources = std::max(pl->max_part_sources,
+                                    (pl->part_off[q + 1] - pl->part_off[q]) + (slot_base[q + 1] - slot_base[q]));
   if (n + pl->H > 0x7FFFFFFFLL) return VARCO_UNSUPPORTED;
 
   // counts and send order
@@ -364,6 +367,12 @@ int varco_partition_info(const varco_plan_t *plan, int64_t *n, int64_t *nnz, int
 int varco_partition_boundary_rows(const varco_plan_t *plan, int64_t *count) {
   if (!plan || !count) return VARCO_INVALID_ARG;
   *count = plan->nb;
+  return VARCO_OK;
+}
+
+int varco_partition_set_l2_budget(varco_plan_t *plan, int64_t bytes) {
+  if (!plan || bytes < 0) return VARCO_INVALID_ARG;
+  plan->l2_budget = bytes;
   return VARCO_OK;
 }
 

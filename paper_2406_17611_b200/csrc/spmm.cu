@@ -708,6 +708,20 @@ int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, cons
   a.nv = nv;
   a.panels = 1;
   a.nv_panel = nv;
+  // Optional feature panels (off unless an L2 budget is set on the plan): split the feature row so that what
+  // one partition gathers from fits the budget.  Measured on this part it does not pay, neither on the
+  // products-like graph (5 uses per source row) nor on the dense one (60 uses): the kernels are bound by
+  // instruction issue at about 6-7 TB/s of gathered bytes, below what L2 could deliver, so the extra index
+  // passes only add work.  Kept as a knob for other graphs and parts.
+  const int64_t footprint = pl->max_part_sources * (int64_t)nv * 16;
+  if (pl->l2_budget > 0 && footprint > pl->l2_budget && nv > 4) {
+    int panels = (int)((footprint + pl->l2_budget - 1) / pl->l2_budget);
+    int nvp = (nv + panels - 1) / panels;
+    nvp = (nvp + 3) / 4 * 4;              // whole 64-byte units
+    if (nvp < 4) nvp = 4;
+    a.nv_panel = nvp;
+    a.panels = (nv + nvp - 1) / nvp;
+  }
   a.short_col = pl->d.short_f_col;
   a.short_val = pl->d.short_f_val;
   return dt == VARCO_F32 ? dispatch<float>(a, st) : dispatch<__nv_bfloat16>(a, st);

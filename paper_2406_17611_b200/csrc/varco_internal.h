@@ -49,6 +49,8 @@ struct varco_profile;  // CUDA-event bookkeeping, defined in runtime.cu
 
 struct varco_plan {
   int64_t n = 0, nnz = 0, nnz_f = 0, H = 0, cross = 0, self_ = 0, nb = 0;
+  int64_t max_part_sources = 0;        // largest (rows + halo slots) of one partition
+  int64_t l2_budget = 0;               // > 0: split feature rows so that a partition's gathered rows fit this many bytes
   int32_t P = 0;
   int conv = 0;
   std::vector<int64_t> new_to_old, part_off, counts, send_base, halo_ids;

@@ -219,6 +219,36 @@ def test_hub_rows(orc, bf16, F_in, F_out):
     plan.close()
 
 
+@pytest.mark.parametrize("bf16,F_in,F_out,conv", [(True, 256, 64, "sage"), (True, 602, 48, "gcn"), (False, 64, 32, "sage")])
+def test_feature_panels_on_dense_graph(orc, bf16, F_in, F_out, conv):
+    """Dense neighbourhoods (about 120 entries per row, every source row reused ~30 times): with a tiny L2
+    budget the forward aggregation runs in its finest feature panels; results must not change."""
+    n, P = 1500, 4
+    rp, col = synth.erdos_renyi(n, 120.0, 21)
+    part = synth.partition_random_equal(n, P, 22)
+    dt = torch.bfloat16 if bf16 else torch.float32
+    rng = np.random.default_rng(5)
+    X = synth.normal_features(n, F_in, 1, bf16)
+    Wn = synth.glorot_uniform(F_in, F_out, 2, bf16)
+    Ws = synth.glorot_uniform(F_in, F_out, 3, bf16) if conv == "sage" else None
+    b = (0.1 * rng.standard_normal(F_out)).astype(np.float32)
+    plan = vb.Plan(rp, col, part, P, conv).upload()
+    plan.set_l2_budget(1024)
+    g = orc.graph(rp, col, part, P, conv)
+    perm = plan.perm()
+    ws = plan.workspace(F_in, F_out, vb.BF16 if bf16 else vb.F32)
+    Xd = to_device_rows(X, perm, dt)
+    for ratio in [(1, 1), (4, 1)]:
+        key = (3, 1, 0)
+        Y, Agg, hb = vb.varco_layer_fwd(plan, Xd, dev_weights(Ws, dt), dev_weights(Wn, dt),
+                                        dev_weights(b, torch.float32), True, ratio, key, ws, F_in=F_in)
+        Yr, Aggr, hbr = g.layer_fwd(X, Ws, Wn, b, True, ratio, key, elem_bytes=2 if bf16 else 4)
+        assert hb == hbr and vb.varco_workspace_status(ws) == 0
+        assert rel_err(to_host_rows(Agg, perm, F_in), Aggr) <= TOL[dt]
+        assert rel_err(to_host_rows(Y, perm, F_out), Yr) <= TOL[dt]
+    plan.close()
+
+
 def test_backward_is_reproducible(cases):
     """The ordered (atomic-free) gradient accumulation gives bit-identical results run to run."""
     case = cases("c2r", 0.05)
