@@ -240,7 +240,7 @@ def stage_work(wl, plan, ratio_k):
         work["decompress"] += H * (k * es + F * es)
         work["spmm"] += nnz_f * 4 + (n + H) * F * es + n * F * es + (n + 1) * 8
         work["spmm_t"] += nnz_f * 4 + n * F * es + (n + H) * F * es + (n + H + 1) * 8
-        work["compress_bwd"] += H * (F * es + k * es)
+        work["compress_bwd"] += plan_nb(plan) * k * 2 if k < F else 0   # 16-bit kept positions, once per boundary row
         work["scatter_add"] += H * k * es + 2 * plan_nb(plan) * F * es
         work["gemm_fwd"] += 2.0 * n * kc * Fo
         work["gemm_dx"] += 2.0 * n * kc * Fo

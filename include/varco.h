@@ -258,7 +258,8 @@ enum {
   VARCO_STAGE_GEMM_DX = 4,       /* dZ W^T                                       */
   VARCO_STAGE_GEMM_DW = 5,       /* [X | Agg]^T dZ and dbias                     */
   VARCO_STAGE_SPMM_T = 6,        /* transposed aggregation (to rows and slots)   */
-  VARCO_STAGE_COMPRESS_BWD = 7,  /* unused: the gradient compression runs in the
+  VARCO_STAGE_COMPRESS_BWD = 7,  /* k < F: kept positions of the boundary rows for the
+                                    backward; the gradient compression itself runs in the
                                     epilogue of the transposed aggregation (stage 6) */
   VARCO_STAGE_SCATTER_ADD = 8,   /* decompress + ordered add into owner rows     */
   VARCO_STAGE_AUX = 9,           /* small helpers: masks, casts, weight repacks  */

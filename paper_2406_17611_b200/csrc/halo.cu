@@ -71,7 +71,8 @@ __global__ void __launch_bounds__(256) compress_rows_kernel(const E *__restrict_
                                                             const int32_t *__restrict__ brow_slot,
                                                             const int32_t *__restrict__ slot_sendpos,
                                                             const int32_t *__restrict__ row_gid, int nb,
-                                                            E *__restrict__ packed, int64_t kstride) {
+                                                            E *__restrict__ packed, int64_t kstride,
+                                                            uint16_t *__restrict__ wpos, int64_t wstride) {
   extern __shared__ uint4 smem_u4[];
   constexpr int V = VecOf<E>::kVec;
   const int nv = (F + V - 1) / V;      // chunks of a row
@@ -92,7 +93,15 @@ __global__ void __launch_bounds__(256) compress_rows_kernel(const E *__restrict_
   init_perm<G>(pm, lkey, (uint32_t)row_gid[r], (uint32_t)F, h, gl, gmask);
   const bool identity = k == F;
   __syncwarp(gmask);
-  for (int m = gl; m < kv * V; m += G) zrow[m] = m < k ? srow[wire_pos(pm, m, identity)] : (E)0;
+  for (int m = gl; m < kv * V; m += G) {
+    E v = (E)0;
+    if (m < k) {
+      const uint32_t p = wire_pos(pm, m, identity);
+      v = srow[p];
+      if (wpos) wpos[(int64_t)r * wstride + m] = (uint16_t)p;   // kept for the receivers of this call
+    }
+    zrow[m] = v;
+  }
   __syncwarp(gmask);
   const bool vec = ((kstride * (int64_t)sizeof(E)) & 15) == 0;
   for (int s = s0; s < s1; ++s) {
@@ -116,7 +125,9 @@ __global__ void __launch_bounds__(256) decompress_slots_kernel(const E *__restri
                                                                int k, int h, uint64_t lkey,
                                                                const int32_t *__restrict__ slot_gid,
                                                                const int32_t *__restrict__ slot_sendpos, int H,
-                                                               E *__restrict__ Xhalo, int64_t ld) {
+                                                               E *__restrict__ Xhalo, int64_t ld,
+                                                               const uint16_t *__restrict__ wpos, int64_t wstride,
+                                                               const int32_t *__restrict__ slot_src) {
   extern __shared__ uint4 smem_u4[];
   constexpr int V = VecOf<E>::kVec;
   const int nv = (F + V - 1) / V;
@@ -139,11 +150,17 @@ __global__ void __launch_bounds__(256) decompress_slots_kernel(const E *__restri
     for (int m = gl; m < k; m += G) zrow[m] = z[m];
   }
   for (int v = gl; v < nv; v += G) srow4[v] = make_uint4(0u, 0u, 0u, 0u);
-  vperm::RowPerm pm;
-  init_perm<G>(pm, lkey, (uint32_t)slot_gid[slot], (uint32_t)F, h, gl, gmask);
-  const bool identity = k == F;
-  __syncwarp(gmask);
-  for (int m = gl; m < k; m += G) srow[wire_pos(pm, m, identity)] = zrow[m];
+  if (wpos) {
+    const uint16_t *prow = wpos + (int64_t)slot_src[slot] * wstride;
+    __syncwarp(gmask);
+    for (int m = gl; m < k; m += G) srow[__ldg(prow + m)] = zrow[m];
+  } else {
+    vperm::RowPerm pm;
+    init_perm<G>(pm, lkey, (uint32_t)slot_gid[slot], (uint32_t)F, h, gl, gmask);
+    const bool identity = k == F;
+    __syncwarp(gmask);
+    for (int m = gl; m < k; m += G) srow[wire_pos(pm, m, identity)] = zrow[m];
+  }
   __syncwarp(gmask);
   uint4 *dst = reinterpret_cast<uint4 *>(Xhalo + (int64_t)slot * ld);
   for (int v = gl; v < nv; v += G) dst[v] = srow4[v];
@@ -154,26 +171,68 @@ __global__ void __launch_bounds__(256) decompress_slots_kernel(const E *__restri
 // received values next to the positions they belong to: pair m = (value m, pi(m)).  The
 // aggregation then reads k pairs per remote neighbour instead of F elements.  bf16: one 32-bit
 // word per pair (value in the low half, position in the high half); fp32: two words.
-template <typename E, int G>
-__global__ void __launch_bounds__(256) expand_slots_kernel(const E *__restrict__ packed, int64_t kstride, int F, int k,
-                                                           int h, uint64_t lkey, const int32_t *__restrict__ slot_gid,
-                                                           int H, uint32_t *__restrict__ pairs, int64_t pstride) {
-  const int slot = (blockIdx.x * blockDim.x + threadIdx.x) / G;
-  const int gl = threadIdx.x % G;
+template <typename E>
+__global__ void __launch_bounds__(256) expand_slots_kernel(const E *__restrict__ packed, int64_t kstride, int k, int H,
+                                                           uint32_t *__restrict__ pairs, int64_t pstride,
+                                                           const uint16_t *__restrict__ wpos, int64_t wstride,
+                                                           const int32_t *__restrict__ slot_src) {
+  // one thread per 16-byte chunk of a packed row: V values and their V positions from the table
+  constexpr int V = VecOf<E>::kVec;
+  const int kv = (int)(kstride / V);
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int slot = (int)(t / kv), c = (int)(t % kv);
   if (slot >= H) return;
-  const unsigned gmask = group_mask<G>();
-  vperm::RowPerm pm;
-  init_perm<G>(pm, lkey, (uint32_t)slot_gid[slot], (uint32_t)F, h, gl, gmask);
-  const E *z = packed + (int64_t)slot * kstride;
-  for (int m = gl; m < pstride; m += G) {
-    const uint32_t pos = m < k ? pm.pi((uint32_t)m) : 0u;
-    const uint32_t v = m < k ? (uint32_t)z[m] : 0u;   // padding pairs: value 0 at position 0
-    if (sizeof(E) == 2) {
-      pairs[(int64_t)slot * pstride + m] = v | (pos << 16);
-    } else {
-      reinterpret_cast<uint2 *>(pairs)[(int64_t)slot * pstride + m] = make_uint2(v, pos);
+  const uint4 z = __ldg(reinterpret_cast<const uint4 *>(packed + (int64_t)slot * kstride) + c);
+  const uint16_t *prow = wpos + (int64_t)__ldg(slot_src + slot) * wstride + c * V;
+  const uint32_t zw[4] = {z.x, z.y, z.z, z.w};
+  uint32_t out[8];
+  if (sizeof(E) == 2) {
+    const uint4 pw = __ldg(reinterpret_cast<const uint4 *>(prow));
+    const uint32_t ps[4] = {pw.x, pw.y, pw.z, pw.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int m = c * 8 + i;
+      const uint32_t v = (zw[i >> 1] >> ((i & 1) * 16)) & 0xFFFFu;
+      const uint32_t pos = (ps[i >> 1] >> ((i & 1) * 16)) & 0xFFFFu;
+      out[i] = m < k ? (v | (pos << 16)) : 0u;   // padding pairs: value 0 at position 0
+    }
+  } else {
+    const uint2 pw = __ldg(reinterpret_cast<const uint2 *>(prow));
+    const uint32_t ps[2] = {pw.x, pw.y};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int m = c * 4 + i;
+      const uint32_t pos = (ps[i >> 1] >> ((i & 1) * 16)) & 0xFFFFu;
+      out[2 * i] = m < k ? zw[i] : 0u;
+      out[2 * i + 1] = m < k ? pos : 0u;
     }
   }
+  // 32 bytes of pairs per chunk; pstride is a multiple of 4 pairs, so a row may end after the first half
+  constexpr int kPairWords = sizeof(E) == 2 ? 1 : 2;
+  uint4 *dst = reinterpret_cast<uint4 *>(pairs + ((int64_t)slot * pstride + (int64_t)c * V) * kPairWords);
+  constexpr int kHalf = V / 2;   // pairs per 16 bytes
+  if (c * V < pstride) dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
+  if (c * V + kHalf < pstride) dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
+}
+
+// ------------------------------------------------------------------------------------------
+// Kept positions of every unique boundary row, evaluated once per call: entry m of table row r is
+// pi_r(m), m < k.  The forward fills the table while compressing; the backward, which runs after
+// other layers have reused the workspace, fills it again from the same key before the kernels
+// that consult it (one evaluation per unique row instead of one per slot copy and per kernel).
+template <int G>
+__global__ void __launch_bounds__(256) wire_positions_kernel(int F, int k, int h, uint64_t lkey,
+                                                             const int32_t *__restrict__ brow,
+                                                             const int32_t *__restrict__ row_gid, int nb,
+                                                             uint16_t *__restrict__ wpos, int64_t wstride) {
+  const int b = (blockIdx.x * blockDim.x + threadIdx.x) / G;
+  const int gl = threadIdx.x % G;
+  if (b >= nb) return;
+  const unsigned gmask = group_mask<G>();
+  const int r = brow[b];
+  vperm::RowPerm pm;
+  init_perm<G>(pm, lkey, (uint32_t)row_gid[r], (uint32_t)F, h, gl, gmask);
+  for (int m = gl; m < k; m += G) wpos[(int64_t)r * wstride + m] = (uint16_t)pm.pi((uint32_t)m);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -182,15 +241,15 @@ __global__ void __launch_bounds__(256) expand_slots_kernel(const E *__restrict__
 // to the owner's gradient row at the kept positions.  No atomics: the result is reproducible.
 template <typename T, int G>
 __global__ void __launch_bounds__(256) scatter_add_rows_kernel(const T *__restrict__ packed, int64_t kstride, int F,
-                                                               int k, int h, uint64_t lkey,
-                                                               const int32_t *__restrict__ brow,
+                                                               int k, const int32_t *__restrict__ brow,
                                                                const int32_t *__restrict__ brow_ptr,
-                                                               const int32_t *__restrict__ brow_slot,
-                                                               const int32_t *__restrict__ row_gid, int nb,
-                                                               T *__restrict__ dX, int64_t ld) {
+                                                               const int32_t *__restrict__ brow_slot, int nb,
+                                                               T *__restrict__ dX, int64_t ld,
+                                                               const uint16_t *__restrict__ wpos, int64_t wstride) {
   extern __shared__ uint4 smem_u4[];
   constexpr int V = ElemTraits<T>::kVec;
   const int nv = (F + V - 1) / V;
+  const int kv = (int)(kstride / V);
   const int grp = threadIdx.x / G, gl = threadIdx.x % G;
   const int b = blockIdx.x * (blockDim.x / G) + grp;
   if (b >= nb) return;
@@ -205,13 +264,45 @@ __global__ void __launch_bounds__(256) scatter_add_rows_kernel(const T *__restri
 #pragma unroll
     for (int i = 0; i < V; ++i) srow[v * V + i] = f[i];
   }
-  vperm::RowPerm pm;
-  init_perm<G>(pm, lkey, (uint32_t)row_gid[r], (uint32_t)F, h, gl, gmask);
   __syncwarp(gmask);
-  for (int m = gl; m < k; m += G) {
-    float sum = 0.f;
-    for (int s = s0; s < s1; ++s) sum += ElemTraits<T>::to_f(packed[(int64_t)brow_slot[s] * kstride + m]);
-    srow[pm.pi((uint32_t)m)] += sum;
+  const uint16_t *prow = wpos + (int64_t)r * wstride;
+  // a lane owns 16-byte chunks of the packed rows: V kept values per load, four slot copies in flight,
+  // summed from zero in ascending slot order, then added at the kept positions (all distinct)
+  for (int v = gl; v < kv; v += G) {
+    float sum[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) sum[i] = 0.f;
+    int s = s0;
+    for (; s + 3 < s1; s += 4) {
+      uint4 q[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        q[u] = __ldg(reinterpret_cast<const uint4 *>(packed + (int64_t)brow_slot[s + u] * kstride) + v);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        float f[V];
+        unpack16(q[u], f, T());
+#pragma unroll
+        for (int i = 0; i < V; ++i) sum[i] += f[i];
+      }
+    }
+    for (; s < s1; ++s) {
+      float f[V];
+      unpack16(__ldg(reinterpret_cast<const uint4 *>(packed + (int64_t)brow_slot[s] * kstride) + v), f, T());
+#pragma unroll
+      for (int i = 0; i < V; ++i) sum[i] += f[i];
+    }
+    uint32_t ps[4];
+    if (V == 8) {
+      const uint4 pw = __ldg(reinterpret_cast<const uint4 *>(prow + v * V));
+      ps[0] = pw.x, ps[1] = pw.y, ps[2] = pw.z, ps[3] = pw.w;
+    } else {
+      const uint2 pw = __ldg(reinterpret_cast<const uint2 *>(prow + v * V));
+      ps[0] = pw.x, ps[1] = pw.y, ps[2] = 0u, ps[3] = 0u;
+    }
+#pragma unroll
+    for (int i = 0; i < V; ++i)
+      if (v * V + i < k) srow[(ps[i >> 1] >> ((i & 1) * 16)) & 0xFFFFu] += sum[i];
   }
   __syncwarp(gmask);
   for (int v = gl; v < nv; v += G) {
@@ -325,7 +416,8 @@ int varco_launch_gather_copy(const varco_plan *pl, const void *X, int64_t ld, in
 
 // send_order != 0: packed rows at the sender's positions (stand-alone entry point), else at the slot
 int varco_launch_compress_rows(const varco_plan *pl, const void *X, int64_t ld, int F, int k, varco_dtype_t dt,
-                               varco_key_t key, void *packed, int64_t kstride, int send_order, cudaStream_t st) {
+                               varco_key_t key, void *packed, int64_t kstride, int send_order, uint16_t *wpos,
+                               int64_t wstride, cudaStream_t st) {
   if (pl->nb == 0) return VARCO_OK;
   const int es = dt == VARCO_F32 ? 4 : 2, V = 16 / es;
   const int nv = (F + V - 1) / V, kv = (k + V - 1) / V;
@@ -336,17 +428,18 @@ int varco_launch_compress_rows(const varco_plan *pl, const void *X, int64_t ld, 
   if (dt == VARCO_F32)
     VARCO_DISPATCH_G(L, (compress_rows_kernel<uint32_t, G><<<L.blocks, L.threads, L.smem, st>>>(
                             (const uint32_t *)X, ld, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot, sp,
-                            pl->d.row_gid, (int)pl->nb, (uint32_t *)packed, kstride)));
+                            pl->d.row_gid, (int)pl->nb, (uint32_t *)packed, kstride, wpos, wstride)));
   else
     VARCO_DISPATCH_G(L, (compress_rows_kernel<uint16_t, G><<<L.blocks, L.threads, L.smem, st>>>(
                             (const uint16_t *)X, ld, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot, sp,
-                            pl->d.row_gid, (int)pl->nb, (uint16_t *)packed, kstride)));
+                            pl->d.row_gid, (int)pl->nb, (uint16_t *)packed, kstride, wpos, wstride)));
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
 int varco_launch_decompress_slots(const varco_plan *pl, const void *packed, int64_t kstride, int send_order, int F,
-                                  int k, varco_dtype_t dt, varco_key_t key, void *Xhalo, int64_t ld, cudaStream_t st) {
+                                  int k, varco_dtype_t dt, varco_key_t key, void *Xhalo, int64_t ld, const uint16_t *wpos,
+                                  int64_t wstride, cudaStream_t st) {
   if (pl->H == 0) return VARCO_OK;
   const int es = dt == VARCO_F32 ? 4 : 2, V = 16 / es;
   const int nv = (F + V - 1) / V, kv = (k + V - 1) / V;
@@ -357,54 +450,66 @@ int varco_launch_decompress_slots(const varco_plan *pl, const void *packed, int6
   if (dt == VARCO_F32)
     VARCO_DISPATCH_G(L, (decompress_slots_kernel<uint32_t, G><<<L.blocks, L.threads, L.smem, st>>>(
                             (const uint32_t *)packed, kstride, F, k, h, lkey, pl->d.slot_gid, sp, (int)pl->H,
-                            (uint32_t *)Xhalo, ld)));
+                            (uint32_t *)Xhalo, ld, wpos, wstride, pl->d.slot_src)));
   else
     VARCO_DISPATCH_G(L, (decompress_slots_kernel<uint16_t, G><<<L.blocks, L.threads, L.smem, st>>>(
                             (const uint16_t *)packed, kstride, F, k, h, lkey, pl->d.slot_gid, sp, (int)pl->H,
-                            (uint16_t *)Xhalo, ld)));
+                            (uint16_t *)Xhalo, ld, wpos, wstride, pl->d.slot_src)));
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
-// packed rows (slot order, stride kstride) -> (value, position) pairs, pstride pairs per slot
-int varco_launch_expand_slots(const varco_plan *pl, const void *packed, int64_t kstride, int F, int k,
-                              varco_dtype_t dt, varco_key_t key, void *pairs, int64_t pstride, cudaStream_t st) {
+// packed rows (slot order, stride kstride) -> (value, position) pairs, pstride pairs per slot; the positions
+// come from the call's table
+int varco_launch_expand_slots(const varco_plan *pl, const void *packed, int64_t kstride, int k, varco_dtype_t dt,
+                              void *pairs, int64_t pstride, const uint16_t *wpos, int64_t wstride, cudaStream_t st) {
   if (pl->H == 0) return VARCO_OK;
-  const int G = k <= 8 ? 8 : (k <= 16 ? 16 : 32);
-  const int h = vperm::half_bits(F);
-  const uint64_t lkey = vperm::layer_key(key);
+  if (!wpos) return VARCO_INVALID_ARG;
+  const int V = dt == VARCO_F32 ? 4 : 8;
   const int threads = 256;
-  const unsigned blocks = (unsigned)(((int64_t)pl->H * G + threads - 1) / threads);
-  HaloLaunch L;
-  L.G = G;
+  const unsigned blocks = (unsigned)(((int64_t)pl->H * (kstride / V) + threads - 1) / threads);
   if (dt == VARCO_F32)
-    VARCO_DISPATCH_G(L, (expand_slots_kernel<uint32_t, G><<<blocks, threads, 0, st>>>(
-                            (const uint32_t *)packed, kstride, F, k, h, lkey, pl->d.slot_gid, (int)pl->H,
-                            (uint32_t *)pairs, pstride)));
+    expand_slots_kernel<uint32_t><<<blocks, threads, 0, st>>>((const uint32_t *)packed, kstride, k, (int)pl->H,
+                                                              (uint32_t *)pairs, pstride, wpos, wstride, pl->d.slot_src);
   else
-    VARCO_DISPATCH_G(L, (expand_slots_kernel<uint16_t, G><<<blocks, threads, 0, st>>>(
-                            (const uint16_t *)packed, kstride, F, k, h, lkey, pl->d.slot_gid, (int)pl->H,
-                            (uint32_t *)pairs, pstride)));
+    expand_slots_kernel<uint16_t><<<blocks, threads, 0, st>>>((const uint16_t *)packed, kstride, k, (int)pl->H,
+                                                              (uint32_t *)pairs, pstride, wpos, wstride, pl->d.slot_src);
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
 int varco_launch_scatter_add_rows(const varco_plan *pl, const void *packed, int64_t kstride, int F, int k,
-                                  varco_dtype_t dt, varco_key_t key, void *dX, int64_t ld, cudaStream_t st) {
+                                  varco_dtype_t dt, void *dX, int64_t ld, const uint16_t *wpos, int64_t wstride,
+                                  cudaStream_t st) {
   if (pl->nb == 0) return VARCO_OK;
+  if (!wpos) return VARCO_INVALID_ARG;
   const int V = dt == VARCO_F32 ? 4 : 8;
   const int nv = (F + V - 1) / V;
   HaloLaunch L = shape(pl->nb, nv, (size_t)nv * V * sizeof(float));
-  const int h = vperm::half_bits(F);
-  const uint64_t lkey = vperm::layer_key(key);
   if (dt == VARCO_F32)
     VARCO_DISPATCH_G(L, (scatter_add_rows_kernel<float, G><<<L.blocks, L.threads, L.smem, st>>>(
-                            (const float *)packed, kstride, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot,
-                            pl->d.row_gid, (int)pl->nb, (float *)dX, ld)));
+                            (const float *)packed, kstride, F, k, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot,
+                            (int)pl->nb, (float *)dX, ld, wpos, wstride)));
   else
     VARCO_DISPATCH_G(L, (scatter_add_rows_kernel<__nv_bfloat16, G><<<L.blocks, L.threads, L.smem, st>>>(
-                            (const __nv_bfloat16 *)packed, kstride, F, k, h, lkey, pl->d.brow, pl->d.brow_ptr,
-                            pl->d.brow_slot, pl->d.row_gid, (int)pl->nb, (__nv_bfloat16 *)dX, ld)));
+                            (const __nv_bfloat16 *)packed, kstride, F, k, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot,
+                            (int)pl->nb, (__nv_bfloat16 *)dX, ld, wpos, wstride)));
+  VARCO_KERNEL_LAUNCHED();
+  return VARCO_OK;
+}
+
+// Kept positions of every unique boundary row of this call (k < F) into the table.
+int varco_launch_wire_positions(const varco_plan *pl, int F, int k, varco_key_t key, uint16_t *wpos, int64_t wstride,
+                                cudaStream_t st) {
+  if (pl->nb == 0) return VARCO_OK;
+  HaloLaunch L;
+  L.G = k <= 8 ? 8 : (k <= 16 ? 16 : 32);
+  const int threads = 256;
+  const unsigned blocks = (unsigned)(((int64_t)pl->nb * L.G + threads - 1) / threads);
+  const int h = vperm::half_bits(F);
+  const uint64_t lkey = vperm::layer_key(key);
+  VARCO_DISPATCH_G(L, (wire_positions_kernel<G><<<blocks, threads, 0, st>>>(F, k, h, lkey, pl->d.brow, pl->d.row_gid,
+                                                                           (int)pl->nb, wpos, wstride)));
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }

@@ -9,7 +9,8 @@
 // workspace carving shared by varco_workspace_bytes and the layer entry points
 struct varco_ws_layout {
   int64_t ld_in = 0, ld_out = 0;  // leading dimensions of the internal buffers
-  size_t status = 0, packed = 0, halo = 0, dZ = 0, dAgg = 0, scratch = 0, scratch_bytes = 0, total = 0;
+  int64_t wstride = 0;            // row stride of the kept-position table (16-bit entries)
+  size_t status = 0, packed = 0, halo = 0, wpos = 0, dZ = 0, dAgg = 0, scratch = 0, scratch_bytes = 0, total = 0;
 };
 varco_ws_layout varco_make_ws_layout(const varco_plan *pl, int F_in, int F_out, varco_dtype_t dt);
 size_t varco_gemm_scratch_bytes(int F_in, int F_out);
@@ -18,13 +19,18 @@ size_t varco_gemm_scratch_bytes(int F_in, int F_out);
 int varco_launch_gather_copy(const varco_plan *pl, const void *X, int64_t ld, int F, varco_dtype_t dt, void *Xhalo,
                              int64_t ldh, cudaStream_t st);
 int varco_launch_compress_rows(const varco_plan *pl, const void *X, int64_t ld, int F, int k, varco_dtype_t dt,
-                               varco_key_t key, void *packed, int64_t kstride, int send_order, cudaStream_t st);
+                               varco_key_t key, void *packed, int64_t kstride, int send_order, uint16_t *wpos,
+                               int64_t wstride, cudaStream_t st);
 int varco_launch_decompress_slots(const varco_plan *pl, const void *packed, int64_t kstride, int send_order, int F,
-                                  int k, varco_dtype_t dt, varco_key_t key, void *Xhalo, int64_t ld, cudaStream_t st);
-int varco_launch_expand_slots(const varco_plan *pl, const void *packed, int64_t kstride, int F, int k,
-                              varco_dtype_t dt, varco_key_t key, void *pairs, int64_t pstride, cudaStream_t st);
+                                  int k, varco_dtype_t dt, varco_key_t key, void *Xhalo, int64_t ld, const uint16_t *wpos,
+                                  int64_t wstride, cudaStream_t st);
+int varco_launch_expand_slots(const varco_plan *pl, const void *packed, int64_t kstride, int k, varco_dtype_t dt,
+                              void *pairs, int64_t pstride, const uint16_t *wpos, int64_t wstride, cudaStream_t st);
 int varco_launch_scatter_add_rows(const varco_plan *pl, const void *packed, int64_t kstride, int F, int k,
-                                  varco_dtype_t dt, varco_key_t key, void *dX, int64_t ld, cudaStream_t st);
+                                  varco_dtype_t dt, void *dX, int64_t ld, const uint16_t *wpos, int64_t wstride,
+                                  cudaStream_t st);
+int varco_launch_wire_positions(const varco_plan *pl, int F, int k, varco_key_t key, uint16_t *wpos, int64_t wstride,
+                                cudaStream_t st);
 int varco_launch_add_dense_rows(const varco_plan *pl, const void *Gh, int64_t ldg, int F, varco_dtype_t dt, void *dX,
                                 int64_t ld, cudaStream_t st);
 // spmm.cu
@@ -32,7 +38,7 @@ int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, cons
                           varco_dtype_t dt, void *Agg, int64_t ldagg, cudaStream_t st);
 int varco_launch_spmm_bwd(const varco_plan *pl, const void *dAgg, int64_t ldd, int F, varco_dtype_t dt, void *dX,
                           int64_t ldx, int accumulate, void *Ghalo, int64_t ldh, void *packed, int64_t kstride, int k,
-                          varco_key_t key, cudaStream_t st);
+                          varco_key_t key, const uint16_t *wpos, int64_t wstride, cudaStream_t st);
 int varco_launch_spmm_fwd_sparse(const varco_plan *pl, const void *X, int64_t ldx, const void *pairs, int64_t pstride,
                                  int k, int F, varco_dtype_t dt, void *Agg, int64_t ldagg, cudaStream_t st);
 bool varco_spmm_sparse_supported(int F, int k, varco_dtype_t dt);

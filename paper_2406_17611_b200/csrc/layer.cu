@@ -56,7 +56,7 @@ int varco_compress(const varco_plan_t *plan, const void *X, int64_t ld, int32_t 
   if (!plan->uploaded) return VARCO_NOT_UPLOADED;
   if (bytes) *bytes = (uint64_t)plan->H * (uint64_t)k * (dtype == VARCO_F32 ? 4u : 2u);
   StageTimer t(plan, VARCO_STAGE_COMPRESS, stream);
-  return varco_launch_compress_rows(plan, X, ld, F, k, dtype, key, packed, k, 1, (cudaStream_t)stream);
+  return varco_launch_compress_rows(plan, X, ld, F, k, dtype, key, packed, k, 1, nullptr, 0, (cudaStream_t)stream);
 }
 
 int varco_decompress(const varco_plan_t *plan, const void *packed, int32_t F, varco_dtype_t dtype, varco_ratio_t c,
@@ -69,7 +69,8 @@ int varco_decompress(const varco_plan_t *plan, const void *packed, int32_t F, va
   if (plan->H > 0 && (!packed || check_matrix(Xhalo, ld, F, V) != VARCO_OK)) return VARCO_INVALID_ARG;
   if (!plan->uploaded) return VARCO_NOT_UPLOADED;
   StageTimer t(plan, VARCO_STAGE_DECOMPRESS, stream);
-  return varco_launch_decompress_slots(plan, packed, k, 1, F, k, dtype, key, Xhalo, ld, (cudaStream_t)stream);
+  return varco_launch_decompress_slots(plan, packed, k, 1, F, k, dtype, key, Xhalo, ld, nullptr, 0,
+                                       (cudaStream_t)stream);
 }
 
 int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, const void *X, const void *W_self,
@@ -94,6 +95,8 @@ int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   char *ws = ws_base(workspace);
   void *packed = ws + L.packed;
   void *Xhalo = ws + L.halo;
+  // kept positions of this call's boundary rows: written by the sender-side kernel, read by the receivers
+  uint16_t *wpos = reinterpret_cast<uint16_t *>(ws + L.wpos);
   int *status = reinterpret_cast<int *>(ws + L.status);
   cudaStream_t st = (cudaStream_t)stream;
   VARCO_CUDA_CHECK(cudaMemsetAsync(status, 0, 256, st));
@@ -113,14 +116,15 @@ int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   } else {
     {
       StageTimer t(plan, VARCO_STAGE_COMPRESS, stream);
-      rc = varco_launch_compress_rows(plan, X, desc->ld_in, F_in, k, dt, key, packed, kstride, 0, st);
+      rc = varco_launch_compress_rows(plan, X, desc->ld_in, F_in, k, dt, key, packed, kstride, 0, wpos, L.wstride, st);
     }
     if (rc != VARCO_OK) return rc;
     StageTimer t(plan, VARCO_STAGE_DECOMPRESS, stream);
     if (sparse)
-      rc = varco_launch_expand_slots(plan, packed, kstride, F_in, k, dt, key, Xhalo, round_up64(k, 4), st);
+      rc = varco_launch_expand_slots(plan, packed, kstride, k, dt, Xhalo, round_up64(k, 4), wpos, L.wstride, st);
     else
-      rc = varco_launch_decompress_slots(plan, packed, kstride, 0, F_in, k, dt, key, Xhalo, L.ld_in, st);
+      rc = varco_launch_decompress_slots(plan, packed, kstride, 0, F_in, k, dt, key, Xhalo, L.ld_in, wpos, L.wstride,
+                                         st);
   }
   if (rc != VARCO_OK) return rc;
   {
@@ -220,7 +224,8 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
     void *Gh = packed;    // [H x ld_out] slot sums of dZ
     {
       StageTimer t(plan, VARCO_STAGE_SPMM_T, stream);
-      rc = varco_launch_spmm_bwd(plan, dZ, lddz, F_out, dt, Gl, L.ld_out, 0, Gh, L.ld_out, nullptr, 0, 0, key, st);
+      rc = varco_launch_spmm_bwd(plan, dZ, lddz, F_out, dt, Gl, L.ld_out, 0, Gh, L.ld_out, nullptr, 0, 0, key, nullptr, 0,
+                                 st);
     }
     if (rc != VARCO_OK) return rc;
     {
@@ -250,11 +255,19 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
     }
   }
   if (rc != VARCO_OK) return rc;
+  // k < F: the kept positions of every unique boundary row are evaluated once, then used by the
+  // compression of the slot gradients and by the owners' add
+  uint16_t *wpos = reinterpret_cast<uint16_t *>(ws + L.wpos);
+  if (k < F_in) {
+    StageTimer t(plan, VARCO_STAGE_COMPRESS_BWD, stream);
+    rc = varco_launch_wire_positions(plan, F_in, k, key, wpos, L.wstride, st);
+    if (rc != VARCO_OK) return rc;
+  }
   {
     StageTimer t(plan, VARCO_STAGE_SPMM_T, stream);
     // k < F: the slot gradients are compressed in the epilogue (no dense slot rows)
     rc = varco_launch_spmm_bwd(plan, dAgg, L.ld_in, F_in, dt, dX, desc->ld_in, sage ? 1 : 0, Ghalo, L.ld_in,
-                               k < F_in ? packed : nullptr, round_up64(k, V), k, key, st);
+                               k < F_in ? packed : nullptr, round_up64(k, V), k, key, wpos, L.wstride, st);
   }
   if (rc != VARCO_OK) return rc;
   // Return of the halo-slot gradients to the owners.  At full communication the slot rows are
@@ -266,7 +279,7 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   const int64_t kstride = round_up64(k, V);
   {
     StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
-    rc = varco_launch_scatter_add_rows(plan, packed, kstride, F_in, k, dt, key, dX, desc->ld_in, st);
+    rc = varco_launch_scatter_add_rows(plan, packed, kstride, F_in, k, dt, dX, desc->ld_in, wpos, L.wstride, st);
   }
   return rc;
 }

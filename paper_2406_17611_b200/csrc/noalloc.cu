@@ -62,8 +62,8 @@ extern "C" int varco_exchange_noalloc(const varco_plan_t *plan, const void *X, i
   int rc = scratch_for_current_device(&packed);
   if (rc != VARCO_OK) return rc;
   // every packed element that decompress reads is written by compress first: nothing to clear
-  rc = varco_launch_compress_rows(plan, X, ld, F, k, dtype, key, packed, kstride, 0, (cudaStream_t)stream);
+  rc = varco_launch_compress_rows(plan, X, ld, F, k, dtype, key, packed, kstride, 0, nullptr, 0, (cudaStream_t)stream);
   if (rc != VARCO_OK) return rc;
-  return varco_launch_decompress_slots(plan, packed, kstride, 0, F, k, dtype, key, Xhalo, ld_halo,
+  return varco_launch_decompress_slots(plan, packed, kstride, 0, F, k, dtype, key, Xhalo, ld_halo, nullptr, 0,
                                        (cudaStream_t)stream);
 }

@@ -226,6 +226,8 @@ varco_ws_layout varco_make_ws_layout(const varco_plan *pl, int F_in, int F_out, 
   L.status = take(256);                             // device status word of the last layer call
   L.packed = take((size_t)pl->H * L.ld_in * es);    // packed rows, stride rounded up to 16 bytes
   L.halo = take((size_t)pl->H * L.ld_in * es);      // forward: decompressed rows; backward: slot gradients
+  L.wstride = round_up64(F_in, 8);
+  L.wpos = take((size_t)pl->n * L.wstride * 2);     // kept positions of the call's boundary rows (k < F)
   L.dZ = take((size_t)pl->n * L.ld_out * es);
   L.dAgg = take((size_t)pl->n * L.ld_in * es);
   L.scratch_bytes = varco_gemm_scratch_bytes(F_in, F_out);

@@ -42,6 +42,9 @@ struct HaloCompress {
   int k, F, h;
   uint64_t lkey;
   const int32_t *slot_gid;
+  const uint16_t *wpos;      // table of kept positions by source row (nullptr: evaluate the permutation here)
+  int64_t wstride;
+  const int32_t *slot_src;
 };
 
 struct SpmmArgs {
@@ -166,12 +169,18 @@ __device__ __forceinline__ void finish_row(float (&acc)[NCH][ElemTraits<T>::kVec
       if (FULL || ch < nv) srow4[ch] = pack16(acc[i], T());
     }
     const int slot = r - dst_split;
+    const E *srow = reinterpret_cast<const E *>(srow4);
+    E *z = reinterpret_cast<E *>(hc.packed) + (int64_t)slot * hc.kstride;
+    if (hc.wpos) {
+      const uint16_t *prow = hc.wpos + (int64_t)__ldg(hc.slot_src + slot) * hc.wstride;
+      __syncwarp(gmask);
+      for (int m = gl; m < (int)hc.kstride; m += G) z[m] = m < hc.k ? srow[__ldg(prow + m)] : (E)0;
+      return;
+    }
     vperm::RowPerm pm;
     if (G >= 8) init_perm<(G >= 8 ? G : 8)>(pm, hc.lkey, (uint32_t)__ldg(hc.slot_gid + slot), (uint32_t)hc.F, hc.h, gl, gmask);
     else pm.init(hc.lkey, (uint32_t)__ldg(hc.slot_gid + slot), (uint32_t)hc.F, hc.h);
     __syncwarp(gmask);
-    const E *srow = reinterpret_cast<const E *>(srow4);
-    E *z = reinterpret_cast<E *>(hc.packed) + (int64_t)slot * hc.kstride;
     for (int m = gl; m < (int)hc.kstride; m += G) z[m] = m < hc.k ? srow[pm.pi((uint32_t)m)] : (E)0;
     return;
   }
@@ -345,10 +354,15 @@ __global__ void __launch_bounds__(256)
     for (int c = threadIdx.x; c < nv; c += blockDim.x) srow4[c] = mine[cnt++];
     __syncthreads();
     const int slot = r - dst_split;
-    vperm::RowPerm pm;
-    pm.init(hc.lkey, (uint32_t)__ldg(hc.slot_gid + slot), (uint32_t)hc.F, hc.h);
     const E *srow = reinterpret_cast<const E *>(srow4);
     E *z = reinterpret_cast<E *>(hc.packed) + (int64_t)slot * hc.kstride;
+    if (hc.wpos) {
+      const uint16_t *prow = hc.wpos + (int64_t)__ldg(hc.slot_src + slot) * hc.wstride;
+      for (int m = threadIdx.x; m < (int)hc.kstride; m += blockDim.x) z[m] = m < hc.k ? srow[__ldg(prow + m)] : (E)0;
+      return;
+    }
+    vperm::RowPerm pm;
+    pm.init(hc.lkey, (uint32_t)__ldg(hc.slot_gid + slot), (uint32_t)hc.F, hc.h);
     for (int m = threadIdx.x; m < (int)hc.kstride; m += blockDim.x) z[m] = m < hc.k ? srow[pm.pi((uint32_t)m)] : (E)0;
     return;
   }
@@ -770,7 +784,7 @@ int varco_launch_spmm_fwd_sparse(const varco_plan *pl, const void *X, int64_t ld
 // key and only the k kept values of every slot are written (slot order, stride kstride).
 int varco_launch_spmm_bwd(const varco_plan *pl, const void *dAgg, int64_t ldd, int F, varco_dtype_t dt, void *dX,
                           int64_t ldx, int accumulate, void *Ghalo, int64_t ldh, void *packed, int64_t kstride, int k,
-                          varco_key_t key, cudaStream_t st) {
+                          varco_key_t key, const uint16_t *wpos, int64_t wstride, cudaStream_t st) {
   const int V = dt == VARCO_F32 ? 4 : 8;
   const int nv = (F + V - 1) / V;
   SpmmArgs a{};
@@ -797,6 +811,8 @@ int varco_launch_spmm_bwd(const varco_plan *pl, const void *dAgg, int64_t ldd, i
   a.nv_panel = nv;
   a.short_col = pl->d.short_t_col;
   a.short_val = pl->d.short_t_val;
-  if (packed) a.hc = HaloCompress{packed, kstride, k, F, vperm::half_bits(F), vperm::layer_key(key), pl->d.slot_gid};
+  if (packed)
+    a.hc = HaloCompress{packed, kstride, k, F, vperm::half_bits(F), vperm::layer_key(key), pl->d.slot_gid, wpos, wstride,
+                        pl->d.slot_src};
   return dt == VARCO_F32 ? dispatch<float>(a, st) : dispatch<__nv_bfloat16>(a, st);
 }
