@@ -236,6 +236,45 @@ __global__ void __launch_bounds__(256) wire_positions_kernel(int F, int k, int h
 }
 
 // ------------------------------------------------------------------------------------------
+// Backward, receiver side, when the slot gradient rows exist densely (they came out of a GEMM):
+// keep the k values at the forward's positions.  One group per slot; positions from the table.
+template <typename E, int G>
+__global__ void __launch_bounds__(256) select_slots_kernel(const E *__restrict__ Gh, int64_t ldg, int nv, int k,
+                                                           int H, E *__restrict__ packed, int64_t kstride,
+                                                           const uint16_t *__restrict__ wpos, int64_t wstride,
+                                                           const int32_t *__restrict__ slot_src) {
+  extern __shared__ uint4 smem_u4[];
+  constexpr int V = VecOf<E>::kVec;
+  const int kv = (int)(kstride / V);
+  const int grp = threadIdx.x / G, gl = threadIdx.x % G;
+  const int slot = blockIdx.x * (blockDim.x / G) + grp;
+  if (slot >= H) return;
+  const unsigned gmask = group_mask<G>();
+  uint4 *srow4 = smem_u4 + (size_t)grp * nv;
+  const E *srow = reinterpret_cast<const E *>(srow4);
+  const uint4 *src = reinterpret_cast<const uint4 *>(Gh + (int64_t)slot * ldg);
+  for (int v = gl; v < nv; v += G) srow4[v] = __ldg(src + v);
+  const uint16_t *prow = wpos + (int64_t)__ldg(slot_src + slot) * wstride;
+  __syncwarp(gmask);
+  uint4 *dst = reinterpret_cast<uint4 *>(packed + (int64_t)slot * kstride);
+  for (int c = gl; c < kv; c += G) {
+    uint32_t ps[4];
+    if (V == 8) {
+      const uint4 pw = __ldg(reinterpret_cast<const uint4 *>(prow + c * V));
+      ps[0] = pw.x, ps[1] = pw.y, ps[2] = pw.z, ps[3] = pw.w;
+    } else {
+      const uint2 pw = __ldg(reinterpret_cast<const uint2 *>(prow + c * V));
+      ps[0] = pw.x, ps[1] = pw.y, ps[2] = 0u, ps[3] = 0u;
+    }
+    E z[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i)
+      z[i] = c * V + i < k ? srow[(ps[i >> 1] >> ((i & 1) * 16)) & 0xFFFFu] : (E)0;
+    dst[c] = *reinterpret_cast<const uint4 *>(z);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Backward, owner side, k < F.  One group per unique boundary row: the packed gradients
 // returned by every destination partition are summed in ascending destination order and added
 // to the owner's gradient row at the kept positions.  No atomics: the result is reproducible.
@@ -494,6 +533,26 @@ int varco_launch_scatter_add_rows(const varco_plan *pl, const void *packed, int6
     VARCO_DISPATCH_G(L, (scatter_add_rows_kernel<__nv_bfloat16, G><<<L.blocks, L.threads, L.smem, st>>>(
                             (const __nv_bfloat16 *)packed, kstride, F, k, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot,
                             (int)pl->nb, (__nv_bfloat16 *)dX, ld, wpos, wstride)));
+  VARCO_KERNEL_LAUNCHED();
+  return VARCO_OK;
+}
+
+// Dense slot gradient rows -> their k kept values (slot order, stride kstride).
+int varco_launch_select_slots(const varco_plan *pl, const void *Gh, int64_t ldg, int F, int k, varco_dtype_t dt,
+                              void *packed, int64_t kstride, const uint16_t *wpos, int64_t wstride, cudaStream_t st) {
+  if (pl->H == 0) return VARCO_OK;
+  if (!wpos) return VARCO_INVALID_ARG;
+  const int V = dt == VARCO_F32 ? 4 : 8;
+  const int nv = (F + V - 1) / V;
+  HaloLaunch L = shape(pl->H, nv, (size_t)nv * 16);
+  if (dt == VARCO_F32)
+    VARCO_DISPATCH_G(L, (select_slots_kernel<uint32_t, G><<<L.blocks, L.threads, L.smem, st>>>(
+                            (const uint32_t *)Gh, ldg, nv, k, (int)pl->H, (uint32_t *)packed, kstride, wpos, wstride,
+                            pl->d.slot_src)));
+  else
+    VARCO_DISPATCH_G(L, (select_slots_kernel<uint16_t, G><<<L.blocks, L.threads, L.smem, st>>>(
+                            (const uint16_t *)Gh, ldg, nv, k, (int)pl->H, (uint16_t *)packed, kstride, wpos, wstride,
+                            pl->d.slot_src)));
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }

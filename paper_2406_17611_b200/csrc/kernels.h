@@ -31,6 +31,8 @@ int varco_launch_scatter_add_rows(const varco_plan *pl, const void *packed, int6
                                   cudaStream_t st);
 int varco_launch_wire_positions(const varco_plan *pl, int F, int k, varco_key_t key, uint16_t *wpos, int64_t wstride,
                                 cudaStream_t st);
+int varco_launch_select_slots(const varco_plan *pl, const void *Gh, int64_t ldg, int F, int k, varco_dtype_t dt,
+                              void *packed, int64_t kstride, const uint16_t *wpos, int64_t wstride, cudaStream_t st);
 int varco_launch_add_dense_rows(const varco_plan *pl, const void *Gh, int64_t ldg, int F, varco_dtype_t dt, void *dX,
                                 int64_t ld, cudaStream_t st);
 // spmm.cu

@@ -215,13 +215,23 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
     if (rc == VARCO_OK && dbias) rc = varco_colsum(n, F_out, dt, dZ, lddz, dbias, scratch, st);
   }
   if (rc != VARCO_OK) return rc;
-  // Narrow backward (full communication, F_out well below F_in, tensor-core path): aggregation and the
-  // weight product commute, so the transposed aggregation runs on the F_out-wide dZ instead of the F_in-wide
-  // dZ W_neigh^T, and the product with W_neigh^T is applied afterwards to the local sums and to the slot sums.
-  const bool narrow = tc && k == F_in && 2 * L.ld_out <= F_in;
+  // Narrow backward (F_out well below F_in, tensor-core path): aggregation and the weight product commute,
+  // so the transposed aggregation runs on the F_out-wide dZ instead of the F_in-wide dZ W_neigh^T, and the
+  // product with W_neigh^T is applied afterwards to the local sums and to the slot sums.  The slot gradient
+  // rows come out of that product densely; with k < F their kept values are selected from them.
+  const bool narrow = tc && 2 * L.ld_out <= F_in;
+  uint16_t *wpos = reinterpret_cast<uint16_t *>(ws + L.wpos);
+  const int64_t kstride = round_up64(k, V);
+  if (k < F_in) {
+    // the kept positions of every unique boundary row are evaluated once, then used by the compression of
+    // the slot gradients and by the owners' add
+    StageTimer t(plan, VARCO_STAGE_COMPRESS_BWD, stream);
+    rc = varco_launch_wire_positions(plan, F_in, k, key, wpos, L.wstride, st);
+    if (rc != VARCO_OK) return rc;
+  }
   if (narrow) {
     void *Gl = dAgg;      // [n x ld_out] local sums of dZ
-    void *Gh = packed;    // [H x ld_out] slot sums of dZ
+    void *Gh = packed;    // [H x ld_out] slot sums of dZ (dead once the slot rows exist)
     {
       StageTimer t(plan, VARCO_STAGE_SPMM_T, stream);
       rc = varco_launch_spmm_bwd(plan, dZ, lddz, F_out, dt, Gl, L.ld_out, 0, Gh, L.ld_out, nullptr, 0, 0, key, nullptr, 0,
@@ -241,8 +251,17 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
                                  scratch, status, st);
     }
     if (rc != VARCO_OK) return rc;
+    if (k == F_in) {
+      StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
+      return varco_launch_add_dense_rows(plan, Ghalo, L.ld_in, F_in, dt, dX, desc->ld_in, st);
+    }
+    {
+      StageTimer t(plan, VARCO_STAGE_COMPRESS_BWD, stream);
+      rc = varco_launch_select_slots(plan, Ghalo, L.ld_in, F_in, k, dt, packed, kstride, wpos, L.wstride, st);
+    }
+    if (rc != VARCO_OK) return rc;
     StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
-    return varco_launch_add_dense_rows(plan, Ghalo, L.ld_in, F_in, dt, dX, desc->ld_in, st);
+    return varco_launch_scatter_add_rows(plan, packed, kstride, F_in, k, dt, dX, desc->ld_in, wpos, L.wstride, st);
   }
   {
     StageTimer t(plan, VARCO_STAGE_GEMM_DX, stream);
@@ -255,19 +274,11 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
     }
   }
   if (rc != VARCO_OK) return rc;
-  // k < F: the kept positions of every unique boundary row are evaluated once, then used by the
-  // compression of the slot gradients and by the owners' add
-  uint16_t *wpos = reinterpret_cast<uint16_t *>(ws + L.wpos);
-  if (k < F_in) {
-    StageTimer t(plan, VARCO_STAGE_COMPRESS_BWD, stream);
-    rc = varco_launch_wire_positions(plan, F_in, k, key, wpos, L.wstride, st);
-    if (rc != VARCO_OK) return rc;
-  }
   {
     StageTimer t(plan, VARCO_STAGE_SPMM_T, stream);
     // k < F: the slot gradients are compressed in the epilogue (no dense slot rows)
     rc = varco_launch_spmm_bwd(plan, dAgg, L.ld_in, F_in, dt, dX, desc->ld_in, sage ? 1 : 0, Ghalo, L.ld_in,
-                               k < F_in ? packed : nullptr, round_up64(k, V), k, key, wpos, L.wstride, st);
+                               k < F_in ? packed : nullptr, kstride, k, key, wpos, L.wstride, st);
   }
   if (rc != VARCO_OK) return rc;
   // Return of the halo-slot gradients to the owners.  At full communication the slot rows are
@@ -276,7 +287,6 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
     StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
     return varco_launch_add_dense_rows(plan, Ghalo, L.ld_in, F_in, dt, dX, desc->ld_in, st);
   }
-  const int64_t kstride = round_up64(k, V);
   {
     StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
     rc = varco_launch_scatter_add_rows(plan, packed, kstride, F_in, k, dt, dX, desc->ld_in, wpos, L.wstride, st);

@@ -744,7 +744,8 @@ int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, cons
 bool varco_spmm_sparse_supported(int F, int k, varco_dtype_t dt) {
   const int V = dt == VARCO_F32 ? 4 : 8;
   const int nv = (F + V - 1) / V;
-  // pays (measured) when a remote row shrinks to at most an eighth; positions must fit the pair format;
+  // pays (measured) when a remote row shrinks to at most an eighth (at a quarter the shared-memory updates cost
+  // more than the halved gathers save); positions must fit the pair format;
   // 32 groups of nv * V floats must fit the default shared-memory window
   return nv <= 64 && 8 * k <= F && F <= 65535 && (size_t)32 * nv * V * sizeof(float) <= 48 * 1024;
 }
