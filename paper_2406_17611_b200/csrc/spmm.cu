@@ -16,7 +16,10 @@
 // stays in L2.  Work is issued partition by partition; the kernels can also split the feature
 // row into panels (task = (partition, panel, row)) so that a partition's gathered set fits in L2,
 // but on the measured workloads the extra passes cost more than the hits return, so the
-// launchers use one panel.
+// launchers use one panel.  Measured and dropped: fetching every gathered row with one bulk asynchronous
+// copy (cp.async.bulk into a per-warp shared-memory ring, mbarrier completion, two or four stages): at
+// 512 bytes per copy the copy path sustained about one row per 25 SM cycles, 1.5x slower than the 128-bit
+// loads used here.
 #include <algorithm>
 
 #include "device_common.cuh"
@@ -100,6 +103,18 @@ struct GatherSrc {
   int split;
 };
 
+// acc[j] = w * f[j] + acc[j] for V values, two per instruction (packed fp32 FMA of sm_100; each half rounds
+// like a scalar fmaf, so results are unchanged)
+template <int V>
+__device__ __forceinline__ void fma_row(float (&acc)[V], float w, const float (&f)[V]) {
+#pragma unroll
+  for (int j = 0; j < V; j += 2)
+    asm("{\n\t.reg .b64 a, b, c, d;\n\tmov.b64 a, {%2, %3};\n\tmov.b64 b, {%4, %4};\n\tmov.b64 c, {%0, %1};\n\t"
+        "fma.rn.f32x2 d, a, b, c;\n\tmov.b64 {%0, %1}, d;\n\t}"
+        : "+f"(acc[j]), "+f"(acc[j + 1])
+        : "f"(f[j]), "f"(f[j + 1]), "f"(w));
+}
+
 // Accumulate `len` entries of one row: acc[i][:] += val[e] * chunk (ch_lo + gl + i G) of source col[e].
 // FULL: the group covers exactly the row's chunks, no bounds test on the chunk index.
 // Entries are taken G at a time; lanes beyond the last entry of a batch hold a valid column with weight
@@ -133,8 +148,7 @@ __device__ __forceinline__ void accumulate_range(const int32_t *__restrict__ col
         for (int i = 0; i < NCH; ++i) {
           float f[V];
           unpack16(v[u][i], f, T());
-#pragma unroll
-          for (int j = 0; j < V; ++j) acc[i][j] = fmaf(w[u], f[j], acc[i][j]);
+          fma_row<V>(acc[i], w[u], f);
         }
     }
   }
@@ -278,8 +292,7 @@ __global__ void __launch_bounds__(256)
       for (int i = 0; i < NCH; ++i) {
         float f[V];
         unpack16(v[u][i], f, T());
-#pragma unroll
-        for (int j = 0; j < V; ++j) acc[i][j] = fmaf(w[u], f[j], acc[i][j]);
+        fma_row<V>(acc[i], w[u], f);
       }
   }
   finish_row<T, G, NCH, FULL>(acc, r, gl, gmask, 0, nv, nv, stage_rows, O0, ldo0, O1, ldo1, dst_split, accumulate0, hc);
