@@ -53,6 +53,8 @@ def stage_of(kernels):
             st = "scatter_add"
         elif k.startswith(("dw_kernel", "dw_reduce", "colsum", "reduce_partials")):
             st = "gemm_dw"
+        elif k.startswith(("wire_positions", "select_slots")):
+            st = "compress_bwd"
         elif k.startswith("relu_mask"):
             st = "aux"
         elif k.startswith("spmm"):
