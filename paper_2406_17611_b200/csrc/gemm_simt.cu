@@ -118,15 +118,20 @@ __global__ void reduce_partials_kernel(const float *__restrict__ partial, int64_
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= count) return;
   float s = 0.f;
+#pragma unroll 16
   for (int z = 0; z < splits; ++z) s += partial[(int64_t)z * count + i];
   out[i] = s;
 }
 
 // partial[z][c] = sum over the rows of chunk z of dZ[row][c].  Block = 32 x 8 threads: x owns a 16-byte
 // chunk of columns, y strides over the rows; the eight row-partials meet in shared memory in y order.
-template <typename T>
+// With MASK the rows summed are dY where Y > 0 (else 0), and they are written to dZ on the way: the ReLU
+// mask of the backward pass and the bias gradient in one pass over dY.
+template <typename T, bool MASK>
 __global__ void __launch_bounds__(256) colsum_kernel(const T *__restrict__ dZ, int64_t ld, int rows, int N, int nv,
-                                                     int row_chunk, float *__restrict__ partial) {
+                                                     int row_chunk, float *__restrict__ partial,
+                                                     const T *__restrict__ Y, int64_t ldy, T *__restrict__ dZout,
+                                                     int64_t ldout) {
   constexpr int V = ElemTraits<T>::kVec;
   __shared__ float red[8][32][V + 1];
   const int ch = blockIdx.x * 32 + threadIdx.x;
@@ -135,11 +140,34 @@ __global__ void __launch_bounds__(256) colsum_kernel(const T *__restrict__ dZ, i
 #pragma unroll
   for (int j = 0; j < V; ++j) s[j] = 0.f;
   if (ch < nv)
-    for (int r = r0 + threadIdx.y; r < r1; r += 8) {
-      float f[V];
-      unpack16(__ldg(reinterpret_cast<const uint4 *>(dZ + (int64_t)r * ld) + ch), f, T());
+    for (int r = r0 + threadIdx.y; r < r1; r += 16) {
+      // two rows in flight, added in row order
+      const bool two = r + 8 < r1;
+      const int rb = two ? r + 8 : r;
+      const uint4 qa = __ldg(reinterpret_cast<const uint4 *>(dZ + (int64_t)r * ld) + ch);
+      const uint4 qb = __ldg(reinterpret_cast<const uint4 *>(dZ + (int64_t)rb * ld) + ch);
+      float fa[V], fb[V];
+      unpack16(qa, fa, T());
+      unpack16(qb, fb, T());
+      if (MASK) {
+        const uint4 ya4 = __ldg(reinterpret_cast<const uint4 *>(Y + (int64_t)r * ldy) + ch);
+        const uint4 yb4 = __ldg(reinterpret_cast<const uint4 *>(Y + (int64_t)rb * ldy) + ch);
+        float ya[V], yb[V];
+        unpack16(ya4, ya, T());
+        unpack16(yb4, yb, T());
 #pragma unroll
-      for (int j = 0; j < V; ++j) s[j] += f[j];
+        for (int j = 0; j < V; ++j) {
+          fa[j] = ya[j] > 0.f ? fa[j] : 0.f;
+          fb[j] = yb[j] > 0.f ? fb[j] : 0.f;
+        }
+        reinterpret_cast<uint4 *>(dZout + (int64_t)r * ldout)[ch] = pack16(fa, T());
+        if (two) reinterpret_cast<uint4 *>(dZout + (int64_t)rb * ldout)[ch] = pack16(fb, T());
+      }
+#pragma unroll
+      for (int j = 0; j < V; ++j) {
+        s[j] += fa[j];
+        if (two) s[j] += fb[j];
+      }
     }
 #pragma unroll
   for (int j = 0; j < V; ++j) red[threadIdx.y][threadIdx.x][j] = s[j];
@@ -199,7 +227,7 @@ size_t varco_simt_dw_scratch_bytes(int F_in, int F_out) {
   int splits = (2 * 148 + tiles - 1) / tiles;
   if (splits < 1) splits = 1;
   size_t a = (size_t)splits * (size_t)F_in * F_out * sizeof(float);
-  size_t b = (size_t)2 * 148 * F_out * sizeof(float);
+  size_t b = (size_t)4 * 148 * F_out * sizeof(float);   // column-sum partials
   return (a > b ? a : b) + 256;
 }
 
@@ -249,24 +277,42 @@ int varco_simt_gemm_dw(int n, int F_in, int F_out, varco_dtype_t dt, const void 
                              scratch, st);
 }
 
-int varco_colsum(int n, int F_out, varco_dtype_t dt, const void *dZ, int64_t lddz, float *out, float *scratch,
-                 cudaStream_t st) {
-  int splits = 2 * 148;
+namespace {
+template <typename T>
+int colsum_t(int n, int F_out, const T *dZ, int64_t lddz, float *out, float *scratch, const T *Y, int64_t ldy,
+             T *dZout, int64_t ldout, cudaStream_t st) {
+  int splits = 4 * 148;
   int chunk = (n + splits - 1) / splits;
   if (chunk < 1) chunk = 1;
   splits = (n + chunk - 1) / chunk;
-  const int V = dt == VARCO_F32 ? 4 : 8;
+  constexpr int V = ElemTraits<T>::kVec;
   const int nv = (F_out + V - 1) / V;
   dim3 grid((nv + 31) / 32, splits), block(32, 8);
-  if (dt == VARCO_F32)
-    colsum_kernel<float><<<grid, block, 0, st>>>((const float *)dZ, lddz, n, F_out, nv, chunk, scratch);
+  if (Y)
+    colsum_kernel<T, true><<<grid, block, 0, st>>>(dZ, lddz, n, F_out, nv, chunk, scratch, Y, ldy, dZout, ldout);
   else
-    colsum_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16 *)dZ, lddz, n, F_out, nv, chunk,
-                                                         scratch);
+    colsum_kernel<T, false><<<grid, block, 0, st>>>(dZ, lddz, n, F_out, nv, chunk, scratch, nullptr, 0, nullptr, 0);
   VARCO_KERNEL_LAUNCHED();
   reduce_partials_kernel<<<(F_out + 255) / 256, 256, 0, st>>>(scratch, F_out, splits, out);
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
+}
+}  // namespace
+
+int varco_colsum(int n, int F_out, varco_dtype_t dt, const void *dZ, int64_t lddz, float *out, float *scratch,
+                 cudaStream_t st) {
+  if (dt == VARCO_F32)
+    return colsum_t<float>(n, F_out, (const float *)dZ, lddz, out, scratch, nullptr, 0, nullptr, 0, st);
+  return colsum_t<__nv_bfloat16>(n, F_out, (const __nv_bfloat16 *)dZ, lddz, out, scratch, nullptr, 0, nullptr, 0, st);
+}
+
+// dZ = dY where Y > 0 (else 0) and out[c] = sum over the rows of dZ[.][c], in one pass over dY and Y
+int varco_relu_mask_colsum(int n, int F_out, varco_dtype_t dt, const void *Y, int64_t ldy, const void *dY, int64_t lddy,
+                           void *dZ, int64_t lddz, float *out, float *scratch, cudaStream_t st) {
+  if (dt == VARCO_F32)
+    return colsum_t<float>(n, F_out, (const float *)dY, lddy, out, scratch, (const float *)Y, ldy, (float *)dZ, lddz, st);
+  return colsum_t<__nv_bfloat16>(n, F_out, (const __nv_bfloat16 *)dY, lddy, out, scratch, (const __nv_bfloat16 *)Y, ldy,
+                                 (__nv_bfloat16 *)dZ, lddz, st);
 }
 
 int varco_relu_mask(int n, int F_out, varco_dtype_t dt, const void *Y, int64_t ldy, const void *dY, int64_t lddy,

@@ -167,6 +167,86 @@ __global__ void __launch_bounds__(256) decompress_slots_kernel(const E *__restri
 }
 
 // ------------------------------------------------------------------------------------------
+// Receiver side of the layer path, walked by source row.  Every destination of one boundary row uses
+// the same kept positions, so a group takes one unique boundary row: the staging row is zeroed once and
+// the copy of every destination is put in place and written out in turn (each copy overwrites exactly
+// the positions of the one before).  A lane owns KPL 16-byte chunks of the packed rows; it reads the
+// positions of its values once per boundary row (16-byte reads of the call's table, kept in registers)
+// and fetches its chunks of several destinations' copies before the first is used, so a copy costs
+// V 16-bit shared-memory stores per chunk, the row's read-out and its stores to the slot.
+template <typename E, int G, int KPL>
+__global__ void __launch_bounds__(256) decompress_brows_kernel(const E *__restrict__ packed, int64_t kstride, int F,
+                                                               int k, const int32_t *__restrict__ brow,
+                                                               const int32_t *__restrict__ brow_ptr,
+                                                               const int32_t *__restrict__ brow_slot, int nb,
+                                                               E *__restrict__ Xhalo, int64_t ld,
+                                                               const uint16_t *__restrict__ wpos, int64_t wstride) {
+  extern __shared__ uint4 smem_u4[];
+  constexpr int V = VecOf<E>::kVec;
+  constexpr int kAhead = KPL == 1 ? 4 : 2;
+  const int nv = (F + V - 1) / V;
+  const int kv = (int)(kstride / V);     // <= G * KPL
+  const int grp = threadIdx.x / G, gl = threadIdx.x % G;
+  const int b = blockIdx.x * (blockDim.x / G) + grp;
+  if (b >= nb) return;
+  const unsigned gmask = group_mask<G>();
+  uint4 *srow4 = smem_u4 + (size_t)grp * nv;
+  E *srow = reinterpret_cast<E *>(srow4);
+  const int r = brow[b];
+  const int s0 = brow_ptr[b], s1 = brow_ptr[b + 1];
+  const uint16_t *prow = wpos + (int64_t)r * wstride;
+  const uint4 *packed4 = reinterpret_cast<const uint4 *>(packed);
+  const int64_t kstride4 = kstride / V;
+  // positions of this lane's values, two per word
+  uint32_t ps[KPL][V / 2];
+#pragma unroll
+  for (int j = 0; j < KPL; ++j) {
+    const int c = gl + j * G;
+    if (V == 8) {
+      const uint4 pw = c < kv ? __ldg(reinterpret_cast<const uint4 *>(prow + c * V)) : make_uint4(0u, 0u, 0u, 0u);
+      ps[j][0] = pw.x, ps[j][1] = pw.y, ps[j][V / 2 - 2] = pw.z, ps[j][V / 2 - 1] = pw.w;
+    } else {
+      const uint2 pw = c < kv ? __ldg(reinterpret_cast<const uint2 *>(prow + c * V)) : make_uint2(0u, 0u);
+      ps[j][0] = pw.x, ps[j][1] = pw.y;
+    }
+  }
+  for (int v = gl; v < nv; v += G) srow4[v] = make_uint4(0u, 0u, 0u, 0u);
+  __syncwarp(gmask);
+  for (int s = s0; s < s1; s += kAhead) {
+    int slot[kAhead];
+    uint4 z[kAhead][KPL];
+#pragma unroll
+    for (int u = 0; u < kAhead; ++u) slot[u] = __ldg(brow_slot + min(s + u, s1 - 1));
+#pragma unroll
+    for (int u = 0; u < kAhead; ++u)
+#pragma unroll
+      for (int j = 0; j < KPL; ++j)
+        z[u][j] = gl + j * G < kv ? __ldg(packed4 + (int64_t)slot[u] * kstride4 + gl + j * G) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int u = 0; u < kAhead; ++u) {
+      if (s + u >= s1) break;
+#pragma unroll
+      for (int j = 0; j < KPL; ++j) {
+        const uint32_t zw[4] = {z[u][j].x, z[u][j].y, z[u][j].z, z[u][j].w};
+        const int m0 = (gl + j * G) * V;
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+          const uint32_t pos = (ps[j][i >> 1] >> ((i & 1) * 16)) & 0xFFFFu;
+          E val;
+          if (sizeof(E) == 2) val = (E)((zw[i >> 1] >> ((i & 1) * 16)) & 0xFFFFu);
+          else val = (E)zw[i];
+          if (m0 + i < k) srow[pos] = val;
+        }
+      }
+      __syncwarp(gmask);
+      uint4 *dst = reinterpret_cast<uint4 *>(Xhalo + (int64_t)slot[u] * ld);
+      for (int v = gl; v < nv; v += G) dst[v] = srow4[v];
+      __syncwarp(gmask);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // Receiver side, sparse form.  Instead of a dense row with F - k zeros, the slot keeps its k
 // received values next to the positions they belong to: pair m = (value m, pi(m)).  The
 // aggregation then reads k pairs per remote neighbour instead of F elements.  bf16: one 32-bit
@@ -271,6 +351,61 @@ __global__ void __launch_bounds__(256) select_slots_kernel(const E *__restrict__
     for (int i = 0; i < V; ++i)
       z[i] = c * V + i < k ? srow[(ps[i >> 1] >> ((i & 1) * 16)) & 0xFFFFu] : (E)0;
     dst[c] = *reinterpret_cast<const uint4 *>(z);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Backward, receiver side, narrow layers in compressed epochs with at most 8 kept entries (bf16).  The
+// gradient row of a halo slot is (slot sum of dZ) W_neigh^T, F_in wide, but only its k kept entries are
+// returned to the owner: entry m is the dot product of the slot's F_out-wide sum with row pi(m) of W_neigh.
+// One thread per slot: the sum is read once into registers, the k positions come as one 16-byte read of the
+// call's table, W_neigh sits in shared memory as F_in rows of bf16 pairs (row stride odd in words, so that
+// the lanes of a warp, which read different rows, spread over the banks), and the 8 packed values of the
+// slot leave as one 16-byte store.  fp32 accumulation, results rounded to bf16 as a GEMM epilogue would.
+// NVO: 16-byte chunks of a row of sums.
+template <int NVO>
+__global__ void __launch_bounds__(256) slot_kept_product_kernel(const uint4 *__restrict__ Gh4, int64_t ldg4, int F_out,
+                                                                const __nv_bfloat16 *__restrict__ W, int F_in, int k,
+                                                                int H, uint4 *__restrict__ packed4,
+                                                                const uint16_t *__restrict__ wpos, int64_t wstride,
+                                                                const int32_t *__restrict__ slot_src) {
+  extern __shared__ uint32_t w_pairs[];
+  constexpr int NW = NVO * 4;          // words (pairs) per row
+  constexpr int kRowWords = NW + 1;
+  const uint16_t *Wbits = reinterpret_cast<const uint16_t *>(W);
+  for (int i = threadIdx.x; i < F_in * NW; i += blockDim.x) {
+    const int f = i / NW, j = i % NW;
+    const uint32_t lo = 2 * j < F_out ? Wbits[(int64_t)f * F_out + 2 * j] : 0u;
+    const uint32_t hi = 2 * j + 1 < F_out ? Wbits[(int64_t)f * F_out + 2 * j + 1] : 0u;
+    w_pairs[f * kRowWords + j] = lo | (hi << 16);
+  }
+  __syncthreads();
+  for (int slot = blockIdx.x * blockDim.x + threadIdx.x; slot < H; slot += gridDim.x * blockDim.x) {
+    const uint4 pw = __ldg(reinterpret_cast<const uint4 *>(wpos + (int64_t)__ldg(slot_src + slot) * wstride));
+    const uint32_t ps[4] = {pw.x, pw.y, pw.z, pw.w};
+    float g[NVO * 8];
+#pragma unroll
+    for (int i = 0; i < NVO; ++i) {
+      float f[8];
+      unpack16(i * 8 < F_out ? __ldg(Gh4 + (int64_t)slot * ldg4 + i) : make_uint4(0u, 0u, 0u, 0u), f, __nv_bfloat16());
+#pragma unroll
+      for (int j = 0; j < 8; ++j) g[i * 8 + j] = i * 8 + j < F_out ? f[j] : 0.f;
+    }
+    float acc[8];
+#pragma unroll
+    for (int m = 0; m < 8; ++m) {
+      acc[m] = 0.f;
+      if (m < k) {
+        const uint32_t *wr = w_pairs + ((ps[m >> 1] >> ((m & 1) * 16)) & 0xFFFFu) * kRowWords;
+#pragma unroll
+        for (int j = 0; j < NW; ++j) {
+          const uint32_t wj = wr[j];
+          acc[m] = fmaf(g[2 * j], __uint_as_float(wj << 16), acc[m]);
+          acc[m] = fmaf(g[2 * j + 1], __uint_as_float(wj & 0xFFFF0000u), acc[m]);
+        }
+      }
+    }
+    packed4[slot] = pack16(acc, __nv_bfloat16());
   }
 }
 
@@ -482,6 +617,25 @@ int varco_launch_decompress_slots(const varco_plan *pl, const void *packed, int6
   if (pl->H == 0) return VARCO_OK;
   const int es = dt == VARCO_F32 ? 4 : 2, V = 16 / es;
   const int nv = (F + V - 1) / V, kv = (k + V - 1) / V;
+  if (wpos && !send_order && kstride % V == 0 && wstride % 8 == 0 && kstride / V <= 2 * group_size(nv)) {
+    // layer path: slot order on the packed side and a table of positions -> walk by source row
+    HaloLaunch B = shape(pl->nb, nv, (size_t)nv * 16);
+    const bool one = kstride / V <= B.G;
+#define VARCO_DBR(E, KPL)                                                                                        \
+  VARCO_DISPATCH_G(B, (decompress_brows_kernel<E, G, KPL><<<B.blocks, B.threads, B.smem, st>>>(                  \
+                          (const E *)packed, kstride, F, k, pl->d.brow, pl->d.brow_ptr, pl->d.brow_slot, (int)pl->nb, \
+                          (E *)Xhalo, ld, wpos, wstride)))
+    if (dt == VARCO_F32) {
+      if (one) VARCO_DBR(uint32_t, 1);
+      else VARCO_DBR(uint32_t, 2);
+    } else {
+      if (one) VARCO_DBR(uint16_t, 1);
+      else VARCO_DBR(uint16_t, 2);
+    }
+#undef VARCO_DBR
+    VARCO_KERNEL_LAUNCHED();
+    return VARCO_OK;
+  }
   HaloLaunch L = shape(pl->H, nv, (size_t)(nv + kv) * 16);
   const int h = vperm::half_bits(F);
   const uint64_t lkey = vperm::layer_key(key);
@@ -553,6 +707,41 @@ int varco_launch_select_slots(const varco_plan *pl, const void *Gh, int64_t ldg,
     VARCO_DISPATCH_G(L, (select_slots_kernel<uint16_t, G><<<L.blocks, L.threads, L.smem, st>>>(
                             (const uint16_t *)Gh, ldg, nv, k, (int)pl->H, (uint16_t *)packed, kstride, wpos, wstride,
                             pl->d.slot_src)));
+  VARCO_KERNEL_LAUNCHED();
+  return VARCO_OK;
+}
+
+// Kept entries of the slot gradient rows straight from the slot sums of a narrow layer (bf16, k <= 8):
+// packed[slot][m] = Gh[slot] . W_neigh[pi(m)], m < k; packed rows of 8 values.
+bool varco_slot_kept_product_supported(int F_in, int F_out, int k, varco_dtype_t dt) {
+  if (dt != VARCO_BF16 || F_out > 64 || k > 8) return false;
+  const int nvo = ((F_out + 7) / 8 + 1) / 2 * 2;
+  return (size_t)F_in * (nvo * 4 + 1) * 4 <= 48 * 1024;
+}
+
+int varco_launch_slot_kept_product(const varco_plan *pl, const void *Gh, int64_t ldg, int F_out, const void *W_neigh,
+                                   int F_in, int k, void *packed, int64_t kstride, const uint16_t *wpos,
+                                   int64_t wstride, cudaStream_t st) {
+  if (pl->H == 0) return VARCO_OK;
+  if (!wpos || !varco_slot_kept_product_supported(F_in, F_out, k, VARCO_BF16) || ldg % 8 != 0 || ldg < F_out ||
+      kstride != 8 || wstride % 8 != 0)
+    return VARCO_INVALID_ARG;
+  const int nvo = ((F_out + 7) / 8 + 1) / 2 * 2;   // 2, 4, 6 or 8 chunks
+  int dev = 0, sms = 148;
+  VARCO_CUDA_CHECK(cudaGetDevice(&dev));
+  VARCO_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const size_t smem = (size_t)F_in * (nvo * 4 + 1) * 4;
+  const int64_t want = (pl->H + 255) / 256;
+  const unsigned grid = (unsigned)(want < (int64_t)sms * 8 ? want : (int64_t)sms * 8);
+#define VARCO_SKP(N)                                                                                               \
+  slot_kept_product_kernel<N><<<grid, 256, smem, st>>>((const uint4 *)Gh, ldg / 8, F_out, (const __nv_bfloat16 *)W_neigh, \
+                                                       F_in, k, (int)pl->H, (uint4 *)packed, wpos, wstride,           \
+                                                       pl->d.slot_src)
+  if (nvo == 2) VARCO_SKP(2);
+  else if (nvo == 4) VARCO_SKP(4);
+  else if (nvo == 6) VARCO_SKP(6);
+  else VARCO_SKP(8);
+#undef VARCO_SKP
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }

@@ -33,6 +33,10 @@ int varco_launch_wire_positions(const varco_plan *pl, int F, int k, varco_key_t 
                                 cudaStream_t st);
 int varco_launch_select_slots(const varco_plan *pl, const void *Gh, int64_t ldg, int F, int k, varco_dtype_t dt,
                               void *packed, int64_t kstride, const uint16_t *wpos, int64_t wstride, cudaStream_t st);
+bool varco_slot_kept_product_supported(int F_in, int F_out, int k, varco_dtype_t dt);
+int varco_launch_slot_kept_product(const varco_plan *pl, const void *Gh, int64_t ldg, int F_out, const void *W_neigh,
+                                   int F_in, int k, void *packed, int64_t kstride, const uint16_t *wpos,
+                                   int64_t wstride, cudaStream_t st);
 int varco_launch_add_dense_rows(const varco_plan *pl, const void *Gh, int64_t ldg, int F, varco_dtype_t dt, void *dX,
                                 int64_t ld, cudaStream_t st);
 // spmm.cu
@@ -55,6 +59,8 @@ int varco_simt_gemm_dw(int n, int F_in, int F_out, varco_dtype_t dt, const void 
                        int64_t lddz, float *dW, float *scratch, cudaStream_t st);
 int varco_colsum(int n, int F_out, varco_dtype_t dt, const void *dZ, int64_t lddz, float *out, float *scratch,
                  cudaStream_t st);
+int varco_relu_mask_colsum(int n, int F_out, varco_dtype_t dt, const void *Y, int64_t ldy, const void *dY, int64_t lddy,
+                           void *dZ, int64_t lddz, float *out, float *scratch, cudaStream_t st);
 int varco_relu_mask(int n, int F_out, varco_dtype_t dt, const void *Y, int64_t ldy, const void *dY, int64_t lddy,
                     void *dZ, int64_t lddz, cudaStream_t st);
 

@@ -195,9 +195,16 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
 
   const void *dZ = dY;
   int64_t lddz = desc->ld_out;
+  bool bias_done = false;
   if (desc->relu) {
+    // the mask and, when asked for, the bias gradient (column sums of the masked rows) in one pass
     StageTimer t(plan, VARCO_STAGE_AUX, stream);
-    rc = varco_relu_mask(n, F_out, dt, Y, desc->ld_out, dY, desc->ld_out, dZbuf, L.ld_out, st);
+    if (dbias) {
+      rc = varco_relu_mask_colsum(n, F_out, dt, Y, desc->ld_out, dY, desc->ld_out, dZbuf, L.ld_out, dbias, scratch, st);
+      bias_done = true;
+    } else {
+      rc = varco_relu_mask(n, F_out, dt, Y, desc->ld_out, dY, desc->ld_out, dZbuf, L.ld_out, st);
+    }
     if (rc != VARCO_OK) return rc;
     dZ = dZbuf;
     lddz = L.ld_out;
@@ -212,7 +219,7 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
       if (rc == VARCO_OK && sage)
         rc = varco_simt_gemm_dw(n, F_in, F_out, dt, X, desc->ld_in, dZ, lddz, dW_self, scratch, st);
     }
-    if (rc == VARCO_OK && dbias) rc = varco_colsum(n, F_out, dt, dZ, lddz, dbias, scratch, st);
+    if (rc == VARCO_OK && dbias && !bias_done) rc = varco_colsum(n, F_out, dt, dZ, lddz, dbias, scratch, st);
   }
   if (rc != VARCO_OK) return rc;
   // Narrow backward (F_out well below F_in, tensor-core path): aggregation and the weight product commute,
@@ -230,6 +237,7 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
     if (rc != VARCO_OK) return rc;
   }
   if (narrow) {
+    const bool kept_product = k < F_in && varco_slot_kept_product_supported(F_in, F_out, k, dt);
     void *Gl = dAgg;      // [n x ld_out] local sums of dZ
     void *Gh = packed;    // [H x ld_out] slot sums of dZ (dead once the slot rows exist)
     {
@@ -246,11 +254,22 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
       else
         rc = varco_tc_gemm_cat_t(n, F_in, F_out, Gl, L.ld_out, nullptr, 0, W_neigh, nullptr, dX, desc->ld_in, scratch,
                                  status, st);
-      if (rc == VARCO_OK && plan->H > 0)
+      if (rc == VARCO_OK && plan->H > 0 && !kept_product)
         rc = varco_tc_gemm_cat_t((int)plan->H, F_in, F_out, Gh, L.ld_out, nullptr, 0, W_neigh, nullptr, Ghalo, L.ld_in,
                                  scratch, status, st);
     }
     if (rc != VARCO_OK) return rc;
+    if (kept_product) {
+      // few kept entries: each one is a dot product with one row of W_neigh; the F_in-wide rows never exist
+      {
+        StageTimer t(plan, VARCO_STAGE_COMPRESS_BWD, stream);
+        rc = varco_launch_slot_kept_product(plan, Gh, L.ld_out, F_out, W_neigh, F_in, k, Ghalo, kstride, wpos, L.wstride,
+                                            st);
+      }
+      if (rc != VARCO_OK) return rc;
+      StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
+      return varco_launch_scatter_add_rows(plan, Ghalo, kstride, F_in, k, dt, dX, desc->ld_in, wpos, L.wstride, st);
+    }
     if (k == F_in) {
       StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
       return varco_launch_add_dense_rows(plan, Ghalo, L.ld_in, F_in, dt, dX, desc->ld_in, st);

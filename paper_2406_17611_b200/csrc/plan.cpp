@@ -267,6 +267,13 @@ int build(varco_plan *pl, int64_t n, const int64_t *rp0, const int32_t *col0, co
     std::vector<int32_t> *lt[3] = {&pl->hub_t, &pl->order_t, &pl->short_t};
     std::vector<int32_t> *stt[3] = {&pl->hub_t_start, &pl->order_t_start, &pl->short_t_start};
     classify(pl->rpT, rows_of_part, lt, stt);
+    // the short class of the transposed direction is walked by record position only: keep its local rows
+    // (results added into dX) in front of its halo slots (results returned to the owners), each part still
+    // partition-major, so that the slots can be handed to a kernel of their own
+    std::stable_partition(pl->short_t.begin(), pl->short_t.end(), [&](int32_t u) { return (int64_t)u < n; });
+    pl->short_t_nlocal = 0;
+    for (int32_t u : pl->short_t) pl->short_t_nlocal += (int64_t)u < n ? 1 : 0;
+    for (int q = 0; q <= P; ++q) pl->short_t_start[q] = q == 0 ? 0 : (int32_t)pl->short_t.size();
   }
   // fixed-size records of the short rows, in class-list order: 8 sources and 8 weights per row
   // (-1 / 0 beyond the row's length).  The short-row kernels find them by thread index alone, so

@@ -73,6 +73,7 @@ struct SpmmArgs {
   HaloCompress hc;
   const int32_t *short_col;   // 8-entry records of the short class (nullptr: walk the CSR)
   const float *short_val;
+  int short_nlocal;           // leading rows of the short class whose result is a local row (the rest: halo slots)
 };
 
 // task id -> (position in the class list, panel); tasks are ordered (partition, panel, row)
@@ -298,6 +299,63 @@ __global__ void __launch_bounds__(256)
   finish_row<T, G, NCH, FULL>(acc, r, gl, gmask, 0, nv, nv, stage_rows, O0, ldo0, O1, ldo1, dst_split, accumulate0, hc);
 }
 
+// Halo-slot rows of the short class in compressed epochs.  Only the k kept positions of a slot's gradient row
+// travel back to the owner, so only those columns of the gathered rows are read: KL lanes per slot, lane m
+// owns kept position m (from the call's table) and adds up its column over the slot's entries in entry
+// order -- the same fp32 operations the dense kernel performs for that column, hence the same bits.
+template <typename T, int KL>
+__global__ void __launch_bounds__(256)
+    spmm_short_kept_kernel(const int32_t *__restrict__ rec_col, const float *__restrict__ rec_val,
+                           const int32_t *__restrict__ rows, int count, const T *__restrict__ A, int64_t lda,
+                           int dst_split, HaloCompress hc) {
+  typedef typename ElemBits<T>::type E;
+  static_assert(KL >= 8, "a record has 8 entries, one per lane");
+  const int task = (blockIdx.x * blockDim.x + threadIdx.x) / KL;
+  const int gl = threadIdx.x % KL;
+  if (task >= count) return;
+  const unsigned lane = threadIdx.x % 32;
+  const unsigned gmask = (KL == 32) ? 0xFFFFFFFFu : (((1u << KL) - 1u) << (lane & ~(unsigned)(KL - 1)));
+  int myc = -1;
+  float myw = 0.f;
+  if (gl < 8) {
+    myc = __ldg(rec_col + (int64_t)task * 8 + gl);
+    myw = __ldg(rec_val + (int64_t)task * 8 + gl);
+  }
+  const int slot = __ldg(rows + task) - dst_split;
+  int pos = 0;
+  if (gl < hc.k) pos = __ldg(hc.wpos + (int64_t)__ldg(hc.slot_src + slot) * hc.wstride + gl);
+  const int cnt = __popc(__ballot_sync(gmask, myc >= 0) & gmask);
+  const int c_first = __shfl_sync(gmask, myc, 0, KL);
+  if (myc < 0) myc = c_first;   // lanes past the row's length: a valid source with weight zero
+  const E *col_base = reinterpret_cast<const E *>(A) + pos;
+  float acc = 0.f;
+  for (int t = 0; t < cnt; t += 4) {
+    E x[4];
+    float w[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int c = __shfl_sync(gmask, myc, t + u, KL);
+      w[u] = __shfl_sync(gmask, myw, t + u, KL);
+      x[u] = __ldg(col_base + (int64_t)c * lda);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      float f;
+      if (sizeof(E) == 2) f = __uint_as_float((uint32_t)x[u] << 16);
+      else f = __uint_as_float((uint32_t)x[u]);
+      acc = fmaf(f, w[u], acc);
+    }
+  }
+  if (gl < (int)hc.kstride) {
+    E out = (E)0;
+    if (gl < hc.k) {
+      const T v = ElemTraits<T>::from_f(acc);
+      out = *reinterpret_cast<const E *>(&v);
+    }
+    reinterpret_cast<E *>(hc.packed)[(int64_t)slot * hc.kstride + gl] = out;
+  }
+}
+
 // Long rows (hubs of a skewed degree distribution): one CTA per (row, panel), every warp takes a
 // contiguous share of the entries, partial sums meet in shared memory and are added in warp order.
 template <typename T, int G, int NCH, int UNR, bool FULL>
@@ -445,19 +503,53 @@ int launch_rows(const SpmmArgs &a, const RowClass &rc, cudaStream_t st) {
 }
 
 template <typename T, int G, int NCH, int UNR>
-int launch_short(const SpmmArgs &a, cudaStream_t st) {
-  if (a.shorts.count == 0) return VARCO_OK;
+int launch_short(const SpmmArgs &a, int first, int count, cudaStream_t st) {
+  if (count == 0) return VARCO_OK;
   const int threads = 256;
-  dim3 grid((unsigned)(((int64_t)a.shorts.count * G + threads - 1) / threads));
+  dim3 grid((unsigned)(((int64_t)count * G + threads - 1) / threads));
   const size_t smem = a.hc.packed ? (size_t)(threads / G) * a.nv * 16 : 0;
+  const int32_t *rc = a.short_col + (int64_t)first * 8;
+  const float *rv = a.short_val + (int64_t)first * 8;
+  const int32_t *rows = a.shorts.rows + first;
   if (a.nv == G * NCH)
     spmm_short_kernel<T, G, NCH, UNR, true><<<grid, threads, smem, st>>>(
-        a.short_col, a.short_val, a.shorts.rows, a.shorts.count, gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1,
-        a.dst_split, a.accumulate0, a.nv, a.hc);
+        rc, rv, rows, count, gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1, a.dst_split, a.accumulate0, a.nv,
+        a.hc);
   else
     spmm_short_kernel<T, G, NCH, UNR, false><<<grid, threads, smem, st>>>(
-        a.short_col, a.short_val, a.shorts.rows, a.shorts.count, gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1,
-        a.dst_split, a.accumulate0, a.nv, a.hc);
+        rc, rv, rows, count, gather_src<T>(a), (T *)a.O0, a.ldo0, (T *)a.O1, a.ldo1, a.dst_split, a.accumulate0, a.nv,
+        a.hc);
+  VARCO_KERNEL_LAUNCHED();
+  return VARCO_OK;
+}
+
+// Reading single columns pays while the k scattered 32-byte sectors of a gathered row are fewer than the
+// sectors of the whole row.
+#ifndef VARCO_KEPT_SECTOR_NUM
+#define VARCO_KEPT_SECTOR_NUM 1
+#define VARCO_KEPT_SECTOR_DEN 1
+#endif
+template <typename T>
+bool kept_columns_pay(const SpmmArgs &a) {
+  if (!a.hc.packed || !a.hc.wpos || a.hc.kstride > 32) return false;
+  return (int64_t)a.hc.k * 32 * VARCO_KEPT_SECTOR_DEN <= (int64_t)a.nv * 16 * VARCO_KEPT_SECTOR_NUM;
+}
+
+template <typename T>
+int launch_short_kept(const SpmmArgs &a, int first, int count, cudaStream_t st) {
+  if (count == 0) return VARCO_OK;
+  const int threads = 256;
+  const int32_t *rc = a.short_col + (int64_t)first * 8;
+  const float *rv = a.short_val + (int64_t)first * 8;
+  const int32_t *rows = a.shorts.rows + first;
+  const int KL = a.hc.kstride <= 8 ? 8 : (a.hc.kstride <= 16 ? 16 : 32);
+  dim3 grid((unsigned)(((int64_t)count * KL + threads - 1) / threads));
+  if (KL == 8)
+    spmm_short_kept_kernel<T, 8><<<grid, threads, 0, st>>>(rc, rv, rows, count, (const T *)a.A0, a.lda0, a.dst_split, a.hc);
+  else if (KL == 16)
+    spmm_short_kept_kernel<T, 16><<<grid, threads, 0, st>>>(rc, rv, rows, count, (const T *)a.A0, a.lda0, a.dst_split, a.hc);
+  else
+    spmm_short_kept_kernel<T, 32><<<grid, threads, 0, st>>>(rc, rv, rows, count, (const T *)a.A0, a.lda0, a.dst_split, a.hc);
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
@@ -468,7 +560,15 @@ template <typename T, int G, int NCH, int UNR, int GS, int NCHS, int UNRS>
 int launch(const SpmmArgs &a, cudaStream_t st) {
   if (int rc = launch_hubs<T, (G < 8 ? 8 : G), (G < 8 ? 1 : NCH), UNR>(a, st)) return rc;
   if (int rc = launch_rows<T, G, NCH, UNR>(a, a.normal, st)) return rc;
-  if (a.panels == 1 && a.short_col) return launch_short<T, (GS < 8 ? 8 : GS), (GS < 8 ? (NCHS * GS + 7) / 8 : NCHS), VARCO_SHORT_UNR>(a, st);
+  if (a.panels == 1 && a.short_col) {
+    constexpr int GR = GS < 8 ? 8 : GS, NR = GS < 8 ? (NCHS * GS + 7) / 8 : NCHS;
+    const int nl = a.short_nlocal, ns = a.shorts.count - nl;
+    if (ns > 0 && kept_columns_pay<T>(a)) {
+      if (int rc = launch_short<T, GR, NR, VARCO_SHORT_UNR>(a, 0, nl, st)) return rc;
+      return launch_short_kept<T>(a, nl, ns, st);
+    }
+    return launch_short<T, GR, NR, VARCO_SHORT_UNR>(a, 0, a.shorts.count, st);
+  }
   return launch_rows<T, GS, NCHS, UNRS>(a, a.shorts, st);
 }
 
@@ -751,6 +851,7 @@ int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, cons
   }
   a.short_col = pl->d.short_f_col;
   a.short_val = pl->d.short_f_val;
+  a.short_nlocal = (int)pl->short_f.size();
   return dt == VARCO_F32 ? dispatch<float>(a, st) : dispatch<__nv_bfloat16>(a, st);
 }
 
@@ -825,6 +926,7 @@ int varco_launch_spmm_bwd(const varco_plan *pl, const void *dAgg, int64_t ldd, i
   a.nv_panel = nv;
   a.short_col = pl->d.short_t_col;
   a.short_val = pl->d.short_t_val;
+  a.short_nlocal = (int)pl->short_t_nlocal;
   if (packed)
     a.hc = HaloCompress{packed, kstride, k, F, vperm::half_bits(F), vperm::layer_key(key), pl->d.slot_gid, wpos, wstride,
                         pl->d.slot_src};

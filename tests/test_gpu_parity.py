@@ -77,7 +77,7 @@ CONFIG_LAYERS = [("c1", 1.0, 0), ("c1", 1.0, 1), ("c2", 0.05, 0), ("c2r", 0.05, 
 
 
 @pytest.mark.parametrize("name,scale,layer", CONFIG_LAYERS)
-@pytest.mark.parametrize("ratio", [(1, 1), (16, 1), (1935, 20)])
+@pytest.mark.parametrize("ratio", [(1, 1), (4, 1), (16, 1), (1935, 20)])
 def test_layer_forward_and_backward(orc, cases, name, scale, layer, ratio):
     case = cases(name, scale)
     wl, dt = case.wl, case.dtype
