@@ -42,18 +42,25 @@ def _short(name):
 
 def stage_of(kernels):
     """Stage of every launch of an epoch, from the order the layer entry points launch their kernels."""
-    stages, seen_fwd_gemm = [], 0
+    stages, seen_fwd_gemm, masked_colsum = [], 0, False
     n_layers = sum(1 for k in kernels if k.startswith("rows_kernel")) // 2
     for k in kernels:
         if k.startswith(("gather_copy", "compress_rows")):
             st = "compress"
-        elif k.startswith(("decompress_slots", "expand_slots")):
+        elif k.startswith(("decompress_slots", "decompress_brows", "expand_slots")):
             st = "decompress"
         elif k.startswith(("add_dense_rows", "scatter_add_rows")):
             st = "scatter_add"
-        elif k.startswith(("dw_kernel", "dw_reduce", "colsum", "reduce_partials")):
+        elif k.startswith("colsum"):
+            # the masked form is the ReLU mask of the backward pass with the bias gradient fused in
+            masked_colsum = "true" in k
+            st = "aux" if masked_colsum else "gemm_dw"
+        elif k.startswith("reduce_partials"):
+            st = "aux" if masked_colsum else "gemm_dw"
+            masked_colsum = False
+        elif k.startswith(("dw_kernel", "dw_reduce")):
             st = "gemm_dw"
-        elif k.startswith(("wire_positions", "select_slots")):
+        elif k.startswith(("wire_positions", "select_slots", "slot_kept_product")):
             st = "compress_bwd"
         elif k.startswith("relu_mask"):
             st = "aux"

@@ -55,24 +55,28 @@ def sample_rows(big, count):
     return np.asarray(sorted(rows), dtype=np.int64)
 
 
-@pytest.mark.parametrize("ratio", [(1, 1), (4, 1), (385, 4)])
-def test_layer_on_sampled_rows(orc, big, ratio):
+@pytest.mark.parametrize("layer,ratio", [(1, (1, 1)), (1, (4, 1)), (1, (385, 4)), (2, (1, 1)), (2, (64, 1)),
+                                         (2, (8, 1))])
+def test_layer_on_sampled_rows(orc, big, layer, ratio):
+    """Layer 1 (256 -> 256, ReLU) and the output layer (256 -> 47, linear: the narrow backward, whose slot
+    gradients come from the kept-entry product at 64:1 and from the product + selection at 8:1)."""
     wl, plan, g, perm, inv, ws = (big[k] for k in ("wl", "plan", "g", "perm", "inv", "ws"))
-    layer, F_in, F_out = 1, 256, 256
+    F_in, F_out = wl.widths[layer], wl.widths[layer + 1]
+    relu = layer < len(wl.widths) - 2
     dt = torch.bfloat16
     Ws, Wn, b = wl.layer_weights(layer)
     X = synth.normal_features(wl.n, F_in, SEED + 1, True)            # original order, bf16-representable
     Xd = torch.from_numpy(X[perm]).to(dt).cuda()
     key = (SEED, 7, layer)
     Y, Agg, hb = vb.varco_layer_fwd(plan, Xd, dev_weights(Ws, dt), dev_weights(Wn, dt),
-                                    dev_weights(b, torch.float32), True, ratio, key, ws, F_in=F_in)
+                                    dev_weights(b, torch.float32), relu, ratio, key, ws, F_in=F_in)
     assert vb.varco_workspace_status(ws) == 0
     k = orc.kept(F_in, ratio)
     assert hb == g.H_total * k * 2
     rows = sample_rows(big, 48)
     X64 = X.astype(np.float64)
-    Yr, Aggr = g.layer_fwd_rows(rows, X64, Ws, Wn, b, True, ratio, key)
-    got_Y = Y[torch.from_numpy(inv[rows]).cuda()].double().cpu().numpy()
+    Yr, Aggr = g.layer_fwd_rows(rows, X64, Ws, Wn, b, relu, ratio, key)
+    got_Y = Y[torch.from_numpy(inv[rows]).cuda()][:, :F_out].double().cpu().numpy()
     got_A = Agg[torch.from_numpy(inv[rows]).cuda()].double().cpu().numpy()
     assert rel_err(got_A, Aggr) <= 2e-2
     assert rel_err(got_Y, Yr) <= 2e-2
@@ -80,18 +84,19 @@ def test_layer_on_sampled_rows(orc, big, ratio):
     # backward on sampled rows; Y fed to both sides is the device's own forward output (its ReLU
     # mask is then the same decision on both sides), dY is seeded
     dY = synth.bf16_round(np.random.default_rng(11).standard_normal((wl.n, F_out)).astype(np.float32))
-    dYd = torch.from_numpy(dY[perm]).to(dt).cuda()
-    dX, dWs, dWn, db, hb2 = vb.varco_layer_bwd(plan, Xd, Y, Agg, dev_weights(Ws, dt), dev_weights(Wn, dt), dYd, True,
+    dYd = torch.zeros_like(Y)
+    dYd[:, :F_out] = torch.from_numpy(dY[perm]).to(dt).cuda()
+    dX, dWs, dWn, db, hb2 = vb.varco_layer_bwd(plan, Xd, Y, Agg, dev_weights(Ws, dt), dev_weights(Wn, dt), dYd, relu,
                                                ratio, key, ws, F_in=F_in)
     assert vb.varco_workspace_status(ws) == 0 and hb2 == hb
     Yh = np.empty((wl.n, F_out), dtype=np.float32)
-    Yh[perm] = Y.float().cpu().numpy()
-    rX = g.layer_dx_rows(rows[:24], Yh, Ws, Wn, dY, True, ratio, key)
+    Yh[perm] = Y[:, :F_out].float().cpu().numpy()
+    rX = g.layer_dx_rows(rows[:24], Yh, Ws, Wn, dY, relu, ratio, key)
     got_dX = dX[torch.from_numpy(inv[rows[:24]]).cuda()].double().cpu().numpy()
     assert rel_err(got_dX, rX) <= 2e-2
     # weight gradients: entries recomputed in fp64 from the device's Agg / X and the masked dY
-    dZ = (dYd.double() * (Y > 0).double())
-    for (a, o) in [(0, 0), (17, 200), (255, 255), (100, 3)]:
+    dZ = dYd.double() * (Y > 0).double() if relu else dYd.double()
+    for (a, o) in [(0, 0), (17, 200 % F_out), (255, F_out - 1), (100, 3)]:
         want_n = float((Agg[:, a].double() * dZ[:, o]).sum().item())
         want_s = float((Xd[:, a].double() * dZ[:, o]).sum().item())
         scale_n = float((Agg[:, a].double().abs() * dZ[:, o].abs()).sum().item())
