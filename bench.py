@@ -179,19 +179,36 @@ class DeviceModel:
         return self._forward(ratio, epoch_idx) + self._backward(ratio, epoch_idx)
 
     def epoch_e2e(self, ratio, epoch_idx):
-        """The same epoch fed from pinned host memory, results read back to the host.  X_0 must arrive before
-        the forward pass starts; the upstream gradient is only needed by the backward pass and the logits are
-        final after the forward pass, so those two copies run on a second stream beside the kernels."""
+        """The same epoch fed from pinned host memory, results read back to the host, as a pipeline: all copies
+        run on a second stream beside the kernels.  The input features of the NEXT step are uploaded into the
+        other of two device buffers while this step computes (one upload per step; a step starts once its own
+        upload, issued during the step before, has landed); the upstream gradient is only needed by the backward
+        pass and the logits are final after the forward pass, so those copies overlap the kernels too."""
         torch = self.torch
         main = torch.cuda.current_stream()
         if not hasattr(self, "_copy_stream"):
             self._copy_stream = torch.cuda.Stream()
+            self._x0 = [self.acts[0], torch.empty_like(self.acts[0])]
+            self._x0_ready = [None, None]      # upload of the buffer has landed (recorded on the copy stream)
+            self._x0_free = [None, None]       # the last step that read the buffer is done (recorded on main)
+            self._turn = 0
         side = self._copy_stream
-        side.wait_stream(main)                      # the previous step has released the buffers
-        self.acts[0].copy_(self.X0_host, non_blocking=True)
+        cur, nxt = self._turn % 2, (self._turn + 1) % 2
+        if self._x0_ready[cur] is None:        # very first step: nothing was prefetched
+            with torch.cuda.stream(side):
+                side.wait_stream(main)
+                self._x0[cur].copy_(self.X0_host, non_blocking=True)
+                self._x0_ready[cur] = side.record_event()
         with torch.cuda.stream(side):
+            if self._x0_free[nxt] is not None:
+                side.wait_event(self._x0_free[nxt])
+            self._x0[nxt].copy_(self.X0_host, non_blocking=True)        # the next step's input
+            self._x0_ready[nxt] = side.record_event()
+            side.wait_stream(main)             # the previous backward pass has released the gradient buffer
             self.grads[self.L].copy_(self.dY_host, non_blocking=True)
             dY_ready = side.record_event()
+        main.wait_event(self._x0_ready[cur])
+        self.acts[0] = self._x0[cur]
         total = self._forward(ratio, epoch_idx)
         fwd_done = main.record_event()
         with torch.cuda.stream(side):
@@ -199,7 +216,9 @@ class DeviceModel:
             self.Y_host.copy_(self.acts[self.L], non_blocking=True)
         main.wait_event(dY_ready)
         total += self._backward(ratio, epoch_idx)
+        self._x0_free[cur] = main.record_event()
         main.wait_stream(side)
+        self._turn += 1
         host = [w["dWn"].cpu() for w in self.W]
         return host
 
@@ -443,6 +462,25 @@ def run_ours(args):
     roof["traffic"] = measured_traffic(args, dom)
     roof["algorithmic"] = work.get(dom)
     roof["per"] = "epoch (all launches of the stage)"
+    if dom in ("spmm", "spmm_t") and all(k == f for k, f in zip(ks, wl.widths[:-1])):
+        # The algorithmic bytes count every source row once (an unbounded cache).  What a cache of the L2's size
+        # can do at best under a simple model: the most used rows of every partition, as many as fit, are read
+        # once, every other row once per use (varco_partition_gather_model).
+        l2 = int(torch.cuda.get_device_properties(device).L2_cache_size)
+        es = 2 if wl.bf16 else 4
+        model_bytes = 0.0
+        nnz_f = wl.nnz + (wl.n if wl.conv == "gcn" else 0)
+        for l in range(L):
+            F = wl.widths[l] if dom == "spmm" or 2 * model.ld[l + 1] > wl.widths[l] else wl.widths[l + 1]
+            row = model._ld(F) * es
+            _, _, rows_read = model.plan.gather_model(l2 // row, transposed=(dom == "spmm_t"))
+            out_rows = wl.n if dom == "spmm" else wl.n + model.plan.H_total
+            model_bytes += rows_read * row + nnz_f * 8 + out_rows * row
+        t_s = d["ms_per_step"] * 1e-3
+        roof["cache_model"] = {"l2_bytes": l2, "bytes": model_bytes, "achieved": model_bytes / t_s / 1e9,
+                               "frac": model_bytes / t_s / 1e9 / pk["hbm_gbs"],
+                               "note": "DRAM bytes if the most used source rows of each partition, L2's size worth, "
+                                       "stayed cached and all others were read once per use"}
 
     # epoch time versus rate
     sweep = {}

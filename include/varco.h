@@ -102,6 +102,16 @@ int varco_partition_boundary_rows(const varco_plan_t *plan, int64_t *count);
  * feature row into panels so that the rows one partition gathers from (its own plus its halo slots) fit in
  * `bytes` of L2.  On B200 this did not pay on the measured workloads; results are unchanged either way. */
 int varco_partition_set_l2_budget(varco_plan_t *plan, int64_t bytes);
+/* Analysis aid (no counterpart in the paper): what the aggregation's row gathers cost under a simple cache model.
+ * The aggregation of a partition reads one source row per stored entry, at random; a source used several times
+ * inside the partition is read from memory once only if it stays cached in between.  The model keeps the
+ * `resident_rows` most used sources of every partition cached (read once each) and reads every other source once
+ * per use.  transposed = 0: forward structure (sources = the partition's rows and halo slots); 1: transposed
+ * structure (sources = the partition's rows of the upstream gradient).  Outputs (any may be NULL), summed over
+ * the partitions: entries = row gathers issued, sources = distinct rows gathered (the traffic of an unbounded
+ * cache), rows_read = rows read from memory under the model.  Multiply by the row size for bytes. */
+int varco_partition_gather_model(const varco_plan_t *plan, int32_t transposed, int64_t resident_rows,
+                                 int64_t *entries, int64_t *sources, int64_t *rows_read);
 /* PxP[p * P + q] = |halo(p->q)| (host array of P*P entries). */
 int varco_partition_counts(const varco_plan_t *plan, int64_t *PxP);
 /* Original ids of halo(p->q), ascending; the pointer stays valid until the plan is destroyed. */

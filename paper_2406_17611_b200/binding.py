@@ -20,7 +20,7 @@ STAGES = ["compress", "decompress", "spmm", "gemm_fwd", "gemm_dx", "gemm_dw", "s
           "scatter_add", "aux"]
 
 EXPORTS = ["varco_status_string", "varco_partition_build", "varco_partition_destroy", "varco_partition_info",
-           "varco_partition_boundary_rows", "varco_partition_set_l2_budget", "varco_partition_counts", "varco_partition_halo", "varco_partition_perm", "varco_partition_device_bytes",
+           "varco_partition_boundary_rows", "varco_partition_set_l2_budget", "varco_partition_gather_model", "varco_partition_counts", "varco_partition_halo", "varco_partition_perm", "varco_partition_device_bytes",
            "varco_partition_upload", "varco_workspace_bytes", "varco_kept", "varco_schedule_linear",
            "varco_compress", "varco_decompress", "varco_layer_fwd", "varco_layer_bwd", "varco_profile_enable",
            "varco_profile_reset", "varco_profile_read", "varco_kernel_launches", "varco_workspace_status",
@@ -67,6 +67,7 @@ def lib():
     L.varco_partition_counts.argtypes = [vp, i64p]
     L.varco_partition_boundary_rows.argtypes = [vp, i64p]
     L.varco_partition_set_l2_budget.argtypes = [vp, C.c_int64]
+    L.varco_partition_gather_model.argtypes = [vp, C.c_int32, C.c_int64, i64p, i64p, i64p]
     L.varco_partition_halo.argtypes = [vp, C.c_int32, C.c_int32, C.POINTER(i64p), i64p]
     L.varco_partition_perm.argtypes = [vp, C.POINTER(i64p)]
     L.varco_partition_device_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
@@ -179,6 +180,14 @@ class Plan:
 
     def set_l2_budget(self, nbytes):
         _check(lib().varco_partition_set_l2_budget(self.h, int(nbytes)), "varco_partition_set_l2_budget")
+
+    def gather_model(self, resident_rows, transposed=False):
+        """(row gathers issued, distinct rows gathered, rows read from memory when the `resident_rows` most used
+        sources of every partition stay cached)."""
+        e, s, r = C.c_int64(), C.c_int64(), C.c_int64()
+        _check(lib().varco_partition_gather_model(self.h, int(bool(transposed)), int(resident_rows), C.byref(e),
+                                                  C.byref(s), C.byref(r)), "varco_partition_gather_model")
+        return int(e.value), int(s.value), int(r.value)
 
     def counts(self):
         out = np.zeros((self.P, self.P), dtype=np.int64)

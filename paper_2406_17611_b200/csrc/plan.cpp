@@ -9,6 +9,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <functional>
 #include <new>
 #include <numeric>
 #include <thread>
@@ -104,6 +105,7 @@ int build(varco_plan *pl, int64_t n, const int64_t *rp0, const int32_t *col0, co
   std::vector<int64_t> slot_base(P + 1, 0);
   for (int q = 0; q < P; ++q) slot_base[q + 1] = slot_base[q] + (int64_t)recv[q].size();
   pl->H = slot_base[P];
+  pl->slot_base = slot_base;
   for (int q = 0; q < P; ++q)
     pl->max_part_sources = std::max(pl->max_part_sources,
                                     (pl->part_off[q + 1] - pl->part_off[q]) + (slot_base[q + 1] - slot_base[q]));
@@ -380,6 +382,40 @@ int varco_partition_boundary_rows(const varco_plan_t *plan, int64_t *count) {
 int varco_partition_set_l2_budget(varco_plan_t *plan, int64_t bytes) {
   if (!plan || bytes < 0) return VARCO_INVALID_ARG;
   plan->l2_budget = bytes;
+  return VARCO_OK;
+}
+
+int varco_partition_gather_model(const varco_plan_t *plan, int32_t transposed, int64_t resident_rows, int64_t *entries,
+                                 int64_t *sources, int64_t *rows_read) {
+  if (!plan || resident_rows < 0) return VARCO_INVALID_ARG;
+  const int64_t n = plan->n;
+  int64_t e_tot = 0, s_tot = 0, r_tot = 0;
+  std::vector<int64_t> use;
+  try {
+    for (int q = 0; q < plan->P; ++q) {
+      use.clear();
+      if (transposed) {
+        for (int64_t r = plan->part_off[q]; r < plan->part_off[q + 1]; ++r) use.push_back(plan->rp[r + 1] - plan->rp[r]);
+      } else {
+        for (int64_t r = plan->part_off[q]; r < plan->part_off[q + 1]; ++r)
+          use.push_back(plan->rpT[r + 1] - plan->rpT[r]);
+        for (int64_t u = n + plan->slot_base[q]; u < n + plan->slot_base[q + 1]; ++u)
+          use.push_back(plan->rpT[u + 1] - plan->rpT[u]);
+      }
+      const size_t keep = (size_t)std::min<int64_t>(resident_rows, (int64_t)use.size());
+      std::nth_element(use.begin(), use.begin() + keep, use.end(), std::greater<int64_t>());
+      for (size_t i = 0; i < use.size(); ++i) {
+        e_tot += use[i];
+        s_tot += use[i] > 0 ? 1 : 0;
+        r_tot += i < keep ? (use[i] > 0 ? 1 : 0) : use[i];
+      }
+    }
+  } catch (const std::bad_alloc &) {
+    return VARCO_NOMEM;
+  }
+  if (entries) *entries = e_tot;
+  if (sources) *sources = s_tot;
+  if (rows_read) *rows_read = r_tot;
   return VARCO_OK;
 }
 

@@ -50,6 +50,7 @@ struct varco_profile;  // CUDA-event bookkeeping, defined in runtime.cu
 struct varco_plan {
   int64_t n = 0, nnz = 0, nnz_f = 0, H = 0, cross = 0, self_ = 0, nb = 0;
   int64_t max_part_sources = 0;        // largest (rows + halo slots) of one partition
+  std::vector<int64_t> slot_base;      // [P + 1] first halo slot of every partition
   int64_t short_t_nlocal = 0;          // leading entries of short_t that are local rows (the rest are halo slots)
   int64_t l2_budget = 0;               // > 0: split feature rows so that a partition's gathered rows fit this many bytes
   int32_t P = 0;

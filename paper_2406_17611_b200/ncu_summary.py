@@ -53,7 +53,7 @@ def stage_of(kernels):
             st = "scatter_add"
         elif k.startswith("colsum"):
             # the masked form is the ReLU mask of the backward pass with the bias gradient fused in
-            masked_colsum = "true" in k
+            masked_colsum = k.replace(" ", "").endswith((",1>", ",true>"))
             st = "aux" if masked_colsum else "gemm_dw"
         elif k.startswith("reduce_partials"):
             st = "aux" if masked_colsum else "gemm_dw"

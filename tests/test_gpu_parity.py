@@ -114,6 +114,37 @@ def test_layer_forward_and_backward(orc, cases, name, scale, layer, ratio):
         assert rel_err(host64(dWs), rWs) <= tol
 
 
+@pytest.mark.parametrize("name,scale,layer", [("c1", 1.0, 0), ("c3", 0.004, 1), ("c3", 0.004, 2), ("c4", 0.02, 0)])
+@pytest.mark.parametrize("ratio", [(4, 3), (2, 1), (9, 1)])
+def test_layer_forward_mild_and_mid_ratios(orc, cases, name, scale, layer, ratio):
+    """Ratios between the cases above: three quarters of a row kept (packed rows wider than two chunks per lane:
+    the slot-by-slot decompression), half, and a ninth (kept columns on the way back for the wide rows)."""
+    case = cases(name, scale)
+    wl, dt = case.wl, case.dtype
+    X, Ws, Wn, b, F_in, F_out, relu = layer_io(case, layer, SEED + 3 * layer)
+    key = (SEED + 1, 5, layer)
+    Xd = to_device_rows(X, case.perm, dt)
+    Wsd, Wnd, bd = dev_weights(Ws, dt), dev_weights(Wn, dt), dev_weights(b, torch.float32)
+    Y, Agg, hb = vb.varco_layer_fwd(case.plan, Xd, Wsd, Wnd, bd, relu, ratio, key, case.ws, F_in=F_in)
+    Yr, Aggr, hbr = case.g.layer_fwd(X, Ws, Wn, b, relu, ratio, key, elem_bytes=case.es)
+    assert hb == hbr
+    tol = TOL[dt]
+    assert rel_err(to_host_rows(Agg, case.perm, F_in), Aggr) <= tol
+    assert rel_err(to_host_rows(Y, case.perm, F_out), Yr) <= tol
+    rng = np.random.default_rng(SEED + 9)
+    dY = rng.standard_normal((wl.n, F_out)).astype(np.float32)
+    if wl.bf16:
+        dY = synth.bf16_round(dY)
+    Yd = to_device_rows(Yr.astype(np.float32), case.perm, dt)
+    dX, dWs, dWn, db, hb2 = vb.varco_layer_bwd(case.plan, Xd, Yd, Agg, Wsd, Wnd, to_device_rows(dY, case.perm, dt),
+                                               relu, ratio, key, case.ws, F_in=F_in)
+    rX, rWs, rWn, rb, _ = case.g.layer_bwd(X, to_host_rows(Yd, case.perm, F_out), Ws, Wn, dY, relu, ratio, key,
+                                           elem_bytes=case.es)
+    assert hb2 == hb and vb.varco_workspace_status(case.ws) == 0
+    assert rel_err(to_host_rows(dX, case.perm, F_in), rX) <= tol
+    assert rel_err(host64(dWn), rWn) <= tol and rel_err(host64(db), rb) <= tol
+
+
 def test_tiny_config_two_layer_epochs(orc, cases):
     """Config 1 end to end: 2-layer GCN over the scheduled epochs 0, 3, 4 (k = 1, 2, 64) and at
     full communication; each layer's input is the previous layer's device output."""

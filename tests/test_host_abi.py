@@ -98,3 +98,23 @@ def test_error_codes():
     assert L.varco_workspace_bytes(plan.h, 4096, 4, 0, C.byref(nbytes)) == -7
     assert L.varco_workspace_bytes(plan.h, 64, 64, 0, C.byref(nbytes)) == 0 and nbytes.value > 0
     plan.close()
+
+
+def test_gather_model_matches_brute_force():
+    """Rows read under the static-residency cache model, against a direct count of (partition, source) uses."""
+    wl = synth.make_workload("c3", 0.004)
+    plan = vb.Plan(wl.row_ptr, wl.col, wl.part, wl.parts, wl.conv)
+    rows = np.repeat(np.arange(wl.n), np.diff(wl.row_ptr))
+    dest = wl.part[rows].astype(np.int64)
+    for transposed in (False, True):
+        src = rows if transposed else wl.col.astype(np.int64)
+        _, cnt = np.unique(dest * wl.n + src, return_counts=True)
+        part_of = np.unique(dest * wl.n + src) // wl.n
+        for keep in (0, 7, 300, 10 ** 9):
+            want = 0
+            for q in range(wl.parts):
+                c = np.sort(cnt[part_of == q])[::-1]
+                want += min(keep, len(c)) + int(c[keep:].sum())
+            e, s_, r = plan.gather_model(keep, transposed)
+            assert (e, s_, r) == (int(cnt.sum()), len(cnt), want)
+    plan.close()
