@@ -31,6 +31,15 @@
 
 namespace {
 
+// Resident CTAs per SM the aggregation kernels are compiled for.  At full size the gathers wait on DRAM, and
+// the bytes in flight per SM decide the rate: for rows of at most 512 bytes (one 16-byte chunk per lane of an
+// ordinary or hub row, at most four per lane of a short row) one more resident CTA than the unconstrained
+// register allocation gives (4 -> 5, short rows 3 -> 4, at the price of a few spilled registers) took 1.7 ms
+// off the 57 ms epoch of the 2.45M-node workload; one more again spills into the inner loop and loses 10 ms.
+// Wider rows keep their registers: forced to the same residency they spill and run at half speed.
+constexpr int rows_blocks_per_sm(int nch) { return nch == 1 ? 5 : 1; }
+constexpr int short_blocks_per_sm(int nch) { return nch <= 4 ? 4 : 1; }
+
 struct RowClass {
   const int32_t *rows;   // row ids, partition-major
   const int32_t *start;  // [P + 1] first position of every partition in `rows`
@@ -217,7 +226,7 @@ __device__ __forceinline__ void finish_row(float (&acc)[NCH][ElemTraits<T>::kVec
 }
 
 template <typename T, int G, int NCH, int UNR, bool FULL>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
     spmm_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col, const float *__restrict__ val,
                 RowClass rc, int P, int panels, int nv_panel, GatherSrc gs, T *__restrict__ O0, int64_t ldo0,
                 T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv, HaloCompress hc) {
@@ -248,7 +257,7 @@ __global__ void __launch_bounds__(256)
 // Short rows (at most 8 entries) from fixed-size records: sources and weights of a row sit at 8 * task, so
 // the gathers start after a single dependent load.
 template <typename T, int G, int NCH, int UNR, bool FULL>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, short_blocks_per_sm(NCH))
     spmm_short_kernel(const int32_t *__restrict__ rec_col, const float *__restrict__ rec_val,
                       const int32_t *__restrict__ rows, int count, GatherSrc gs, T *__restrict__ O0, int64_t ldo0,
                       T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv, HaloCompress hc) {
@@ -359,7 +368,7 @@ __global__ void __launch_bounds__(256)
 // Long rows (hubs of a skewed degree distribution): one CTA per (row, panel), every warp takes a
 // contiguous share of the entries, partial sums meet in shared memory and are added in warp order.
 template <typename T, int G, int NCH, int UNR, bool FULL>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
     spmm_hub_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col, const float *__restrict__ val,
                     RowClass rc, int P, int panels, int nv_panel, GatherSrc gs, T *__restrict__ O0, int64_t ldo0,
                     T *__restrict__ O1, int64_t ldo1, int dst_split, int accumulate0, int nv, HaloCompress hc) {
