@@ -661,7 +661,7 @@ __device__ __forceinline__ void accumulate_sparse(const int32_t *__restrict__ co
 
 // One group per row (normal and short classes).  Shared memory: F floats per group.
 template <typename T, int G, int NCH, bool FULL>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
     spmm_sparse_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ nloc,
                        const int32_t *__restrict__ col, const float *__restrict__ val, RowClass rc, GatherSrc gs,
                        const typename SparsePair<T>::type *__restrict__ pairs, int64_t pstride, int k,
@@ -702,7 +702,7 @@ __global__ void __launch_bounds__(256)
 // Hubs: one CTA per row; every warp takes a contiguous share of the local and of the halo entries and
 // owns one shared-memory row; the rows are added in warp order.
 template <typename T, int NCH, bool FULL>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
     spmm_sparse_hub_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ nloc,
                            const int32_t *__restrict__ col, const float *__restrict__ val, RowClass rc, GatherSrc gs,
                            const typename SparsePair<T>::type *__restrict__ pairs, int64_t pstride, int k,
