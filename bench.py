@@ -245,7 +245,8 @@ def measured_traffic(args, stage):
 
 
 def stage_work(wl, plan, ratio_k):
-    """Algorithmic bytes / flops of every stage for ONE epoch (all layers), as the design doc derives."""
+    """Algorithmic bytes / flops of every stage for ONE epoch (all layers): what the method has to move or
+    multiply, every source row counted once."""
     n, nnz, H = wl.n, plan.nnz, plan.H_total
     nnz_f = nnz + (n if wl.conv == "gcn" else 0)
     es = 2 if wl.bf16 else 4
