@@ -230,14 +230,18 @@ int build(varco_plan *pl, int64_t n, const int64_t *rp0, const int32_t *col0, co
     for (int64_t s = 0; s < pl->H; ++s) pl->brow_slot[fill[where[pl->slot_src[s]]]++] = (int32_t)s;
   }
 
-  // processing orders: three classes of rows by number of entries.  Hubs (more than kHubEntries)
+  // processing orders: three classes of rows by number of entries.  Hubs (more than the hub threshold)
   // get a CTA each.  Short rows (at most kShortEntries) are processed by narrow lane groups, several
   // rows per warp.  The rest get a full-width group.  Every class list is partition-major (the
   // kernels sweep partition by partition so that a partition's gathered rows stay in L2) and, inside
   // a partition, sorted by length, longest first, so that the lanes of a warp run alike.
-  const int64_t kHubEntries = 512, kShortEntries = 8;   // the record format below holds 8 entries
+  // The hub threshold differs by direction (measured on the 2.45M-node power-law workload): forward, where the
+  // hub rows sit in one partition and gather from its whole source set, a warp per row serves rows of up to
+  // 2048 entries better than a CTA each (forward stage 18.9 -> 18.2 ms); transposed, where the sources are one
+  // partition's L2-resident block, 512 is the better cut (17.8 ms against 18.4 at 2048).
+  const int64_t kHubEntriesFwd = 2048, kHubEntriesBwd = 512, kShortEntries = 8;   // a record holds 8 entries
   auto classify = [&](const std::vector<int64_t> &ptr, const std::vector<std::vector<int32_t>> &rows_of_part,
-                      std::vector<int32_t> *lists[3], std::vector<int32_t> *starts[3]) {
+                      int64_t kHubEntries, std::vector<int32_t> *lists[3], std::vector<int32_t> *starts[3]) {
     for (int c = 0; c < 3; ++c) {
       lists[c]->clear();
       starts[c]->assign(1, 0);
@@ -263,12 +267,12 @@ int build(varco_plan *pl, int64_t n, const int64_t *rp0, const int32_t *col0, co
       for (int64_t r = pl->part_off[q]; r < pl->part_off[q + 1]; ++r) rows_of_part[q].push_back((int32_t)r);
     std::vector<int32_t> *lf[3] = {&pl->hub_f, &pl->order_f, &pl->short_f};
     std::vector<int32_t> *sf[3] = {&pl->hub_f_start, &pl->order_f_start, &pl->short_f_start};
-    classify(pl->rp, rows_of_part, lf, sf);
+    classify(pl->rp, rows_of_part, kHubEntriesFwd, lf, sf);
     for (int q = 0; q < P; ++q)
       for (int64_t u = n + slot_base[q]; u < n + slot_base[q + 1]; ++u) rows_of_part[q].push_back((int32_t)u);
     std::vector<int32_t> *lt[3] = {&pl->hub_t, &pl->order_t, &pl->short_t};
     std::vector<int32_t> *stt[3] = {&pl->hub_t_start, &pl->order_t_start, &pl->short_t_start};
-    classify(pl->rpT, rows_of_part, lt, stt);
+    classify(pl->rpT, rows_of_part, kHubEntriesBwd, lt, stt);
     // the short class of the transposed direction is walked by record position only: keep its local rows
     // (results added into dX) in front of its halo slots (results returned to the owners), each part still
     // partition-major, so that the slots can be handed to a kernel of their own
