@@ -279,6 +279,11 @@ int varco_profile_enable(varco_plan_t *plan, int on);
 int varco_profile_reset(varco_plan_t *plan);
 int varco_profile_read(varco_plan_t *plan, int64_t *launches /* [VARCO_STAGE_COUNT] */,
                        double *milliseconds /* [VARCO_STAGE_COUNT] */);
+/* The individual timed executions of one stage since the last reset, in the order they were enqueued
+ * (one per layer call that ran the stage): up to `capacity` durations in milliseconds are written to
+ * `milliseconds`, `count` receives how many exist.  Synchronises the events it reads. */
+int varco_profile_spans(varco_plan_t *plan, int32_t stage, double *milliseconds, int64_t capacity,
+                        int64_t *count);
 /* Number of CUDA kernels this library has launched in this process so far (all plans, all
  * streams).  Also a measurement aid without a counterpart in the paper. */
 int varco_kernel_launches(int64_t *count);

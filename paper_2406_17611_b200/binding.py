@@ -23,7 +23,7 @@ EXPORTS = ["varco_status_string", "varco_partition_build", "varco_partition_dest
            "varco_partition_boundary_rows", "varco_partition_set_l2_budget", "varco_partition_gather_model", "varco_partition_counts", "varco_partition_halo", "varco_partition_perm", "varco_partition_device_bytes",
            "varco_partition_upload", "varco_workspace_bytes", "varco_kept", "varco_schedule_linear",
            "varco_compress", "varco_decompress", "varco_layer_fwd", "varco_layer_bwd", "varco_profile_enable",
-           "varco_profile_reset", "varco_profile_read", "varco_kernel_launches", "varco_workspace_status",
+           "varco_profile_reset", "varco_profile_read", "varco_profile_spans", "varco_kernel_launches", "varco_workspace_status",
            "varco_exchange_noalloc"]
 
 
@@ -86,6 +86,7 @@ def lib():
     L.varco_profile_enable.argtypes = [vp, C.c_int]
     L.varco_profile_reset.argtypes = [vp]
     L.varco_profile_read.argtypes = [vp, i64p, C.POINTER(C.c_double)]
+    L.varco_profile_spans.argtypes = [vp, C.c_int32, C.POINTER(C.c_double), C.c_int64, i64p]
     L.varco_kernel_launches.argtypes = [i64p]
     L.varco_workspace_status.argtypes = [vp, vp, i32p]
     _lib = L
@@ -243,6 +244,15 @@ class Plan:
         ms = (C.c_double * n)()
         _check(lib().varco_profile_read(self.h, launches, ms), "varco_profile_read")
         return {STAGES[i]: (int(launches[i]), float(ms[i])) for i in range(n)}
+
+    def profile_spans(self, stage):
+        """Durations (ms) of the individual timed executions of one stage, in enqueue order."""
+        idx = STAGES.index(stage)
+        count = C.c_int64()
+        _check(lib().varco_profile_spans(self.h, idx, None, 0, C.byref(count)), "varco_profile_spans")
+        buf = (C.c_double * max(1, count.value))()
+        _check(lib().varco_profile_spans(self.h, idx, buf, count.value, C.byref(count)), "varco_profile_spans")
+        return [float(buf[i]) for i in range(count.value)]
 
 
 def _dtype_of(t):

@@ -143,7 +143,7 @@ __device__ __forceinline__ uint4 pack16(const float (&f)[8], __nv_bfloat16) {
 template <int G> __device__ __forceinline__ unsigned group_mask() {
   if (G == 32) return 0xFFFFFFFFu;
   const unsigned lane = threadIdx.x & 31u;
-  return ((1u << G) - 1u) << (lane & ~(unsigned)(G - 1));
+  return ((1u << (G & 31)) - 1u) << (lane & ~(unsigned)(G - 1));
 }
 
 // Round keys of one row, computed by six lanes of the group and shared by shuffle (G >= 8).

@@ -186,6 +186,18 @@ int build(varco_plan *pl, int64_t n, const int64_t *rp0, const int32_t *col0, co
     }
   });
 
+  // mean aggregation: every entry of row r carries the same weight 1 / deg(r); the sum kernels add the
+  // sources unweighted and apply it once per row
+  pl->row_scale.clear();
+  if (!gcn) {
+    pl->row_scale.resize(n);
+    for (int64_t r = 0; r < n; ++r) {
+      const int64_t i = pl->new_to_old[r];
+      const double di = (double)(rp0[i + 1] - rp0[i]);
+      pl->row_scale[r] = di > 0 ? (float)(1.0 / di) : 0.f;
+    }
+  }
+
   // number of leading entries of every row whose source is a local row (columns are sorted: local first)
   pl->nloc.resize(n);
   for (int64_t r = 0; r < n; ++r) {

@@ -25,6 +25,7 @@ std::vector<ImageItem> image_items(varco_plan *pl) {
           item(pl->nloc, &d.nloc),
           item(pl->col, &d.col),
           item(pl->val, &d.val),
+          item(pl->row_scale, &d.row_scale),
           item(pl->rpT, &d.rpT),
           item(pl->colT, &d.colT),
           item(pl->valT, &d.valT),
@@ -161,6 +162,27 @@ int varco_profile_read(varco_plan_t *plan, int64_t *launches, double *millisecon
       launches[s] += 1;
       milliseconds[s] += (double)ms;
     }
+  return VARCO_OK;
+}
+
+int varco_profile_spans(varco_plan_t *plan, int32_t stage, double *milliseconds, int64_t capacity, int64_t *count) {
+  if (!plan || !count || stage < 0 || stage >= VARCO_STAGE_COUNT || capacity < 0 || (capacity > 0 && !milliseconds))
+    return VARCO_INVALID_ARG;
+  *count = 0;
+  varco_profile *pr = plan->prof;
+  if (!pr) return VARCO_OK;
+  std::lock_guard<std::mutex> lock(pr->mu);
+  int64_t i = 0;
+  for (auto &sp : pr->spans[stage]) {
+    if (i < capacity) {
+      VARCO_CUDA_CHECK(cudaEventSynchronize(sp.b));
+      float ms = 0.f;
+      VARCO_CUDA_CHECK(cudaEventElapsedTime(&ms, sp.a, sp.b));
+      milliseconds[i] = (double)ms;
+    }
+    ++i;
+  }
+  *count = i;
   return VARCO_OK;
 }
 

@@ -175,6 +175,29 @@ __device__ __forceinline__ uint4 *dest_row(int r, T *O0, int64_t ldo0, T *O1, in
   return reinterpret_cast<uint4 *>(O1 + (int64_t)(r - dst_split) * ldo1);
 }
 
+// Packed row of one slot from its staged gradient row: z[m] = srow[pos[m]], m < k, zeros up to kstride.  Works in
+// 16-byte chunks: a lane reads V positions of the table with one load, picks V elements from shared memory and
+// writes them with one store (the table rows and the packed rows are 16-byte aligned, kstride a multiple of V).
+template <int V>
+__device__ __forceinline__ uint4 load_positions(const uint16_t *__restrict__ prow, int c) {
+  if (V == 8) return __ldg(reinterpret_cast<const uint4 *>(prow + c * V));
+  const uint2 pw = __ldg(reinterpret_cast<const uint2 *>(prow + c * V));
+  return make_uint4(pw.x, pw.y, 0u, 0u);
+}
+template <typename E, int V>
+__device__ __forceinline__ void pick_kept(const E *srow, const uint16_t *__restrict__ prow, E *__restrict__ z, int k,
+                                          int kstride, int lane, int lanes) {
+  uint4 *z4 = reinterpret_cast<uint4 *>(z);
+  for (int c = lane; c * V < kstride; c += lanes) {
+    const uint4 pw = load_positions<V>(prow, c);
+    const uint32_t ps[4] = {pw.x, pw.y, pw.z, pw.w};
+    E out[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) out[i] = c * V + i < k ? srow[(ps[i >> 1] >> ((i & 1) * 16)) & 0xFFFFu] : (E)0;
+    z4[c] = *reinterpret_cast<const uint4 *>(out);
+  }
+}
+
 // Write one finished row: dense (optionally added to what is there), or -- for a halo-slot gradient row of
 // the transposed pass when hc.packed is set -- compressed with the forward's key.
 template <typename T, int G, int NCH, bool FULL>
@@ -198,7 +221,7 @@ __device__ __forceinline__ void finish_row(float (&acc)[NCH][ElemTraits<T>::kVec
     if (hc.wpos) {
       const uint16_t *prow = hc.wpos + (int64_t)__ldg(hc.slot_src + slot) * hc.wstride;
       __syncwarp(gmask);
-      for (int m = gl; m < (int)hc.kstride; m += G) z[m] = m < hc.k ? srow[__ldg(prow + m)] : (E)0;
+      pick_kept<E, V>(srow, prow, z, hc.k, (int)hc.kstride, gl, G);
       return;
     }
     vperm::RowPerm pm;
@@ -438,7 +461,7 @@ __global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
     E *z = reinterpret_cast<E *>(hc.packed) + (int64_t)slot * hc.kstride;
     if (hc.wpos) {
       const uint16_t *prow = hc.wpos + (int64_t)__ldg(hc.slot_src + slot) * hc.wstride;
-      for (int m = threadIdx.x; m < (int)hc.kstride; m += blockDim.x) z[m] = m < hc.k ? srow[__ldg(prow + m)] : (E)0;
+      pick_kept<E, V>(srow, prow, z, hc.k, (int)hc.kstride, (int)threadIdx.x, (int)blockDim.x);
       return;
     }
     vperm::RowPerm pm;
@@ -594,6 +617,245 @@ int dispatch(const SpmmArgs &a, cudaStream_t st) {
   if (w <= 96) return launch<T, 32, 3, 4, 16, 6, 1>(a, st);
   if (w <= 128) return launch<T, 32, 4, 2, 32, 4, 1>(a, st);
   if (w <= 256) return launch<T, 32, 8, 2, 32, 8, 1>(a, st);
+  return VARCO_UNSUPPORTED;
+}
+
+// ------------------------------------------------------------------------------------------
+// Forward mean aggregation as unweighted sums.  Every entry of row i carries the same weight 1 / deg(i), so the
+// source rows are added as they are and the finished row is scaled once.  Per entry the inner loop is one index
+// broadcast, one multiply-add for the address, one 16-byte load and one add per element; a bf16 element goes
+// into its fp32 accumulator with a single mixed-precision add of sm_100 (add.rn.f32.bf16: the bf16 operand is
+// widened exactly and the sum rounded once, the result of widening first).  A row walks its local entries
+// against X and its halo entries against the slot rows in two loops, so no entry needs a base select, and no
+// lane ever multiplies a source by a padding weight of zero (a non-finite source row stays where it belongs).
+__device__ __forceinline__ void add_chunk(float (&acc)[8], const uint4 &v, __nv_bfloat16) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j)
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}"
+        : "+f"(acc[2 * j]), "+f"(acc[2 * j + 1])
+        : "r"(w[j]));
+}
+__device__ __forceinline__ void add_chunk(float (&acc)[4], const uint4 &v, float) {
+  asm("{\n\t.reg .b64 a, c, d;\n\tmov.b64 a, {%2, %3};\n\tmov.b64 c, {%0, %1};\n\tadd.rn.f32x2 d, a, c;\n\t"
+      "mov.b64 {%0, %1}, d;\n\t}"
+      : "+f"(acc[0]), "+f"(acc[1])
+      : "r"(v.x), "r"(v.y));
+  asm("{\n\t.reg .b64 a, c, d;\n\tmov.b64 a, {%2, %3};\n\tmov.b64 c, {%0, %1};\n\tadd.rn.f32x2 d, a, c;\n\t"
+      "mov.b64 {%0, %1}, d;\n\t}"
+      : "+f"(acc[2]), "+f"(acc[3])
+      : "r"(v.z), "r"(v.w));
+}
+
+// acc[i][:] += chunk (gl + i G) of every source col[e], e < len; `base` is the lane's own chunk of row 0
+template <typename T, int G, int NCH, int UNR, bool FULL>
+__device__ __forceinline__ void sum_range(const int32_t *__restrict__ colp, int len, const uint4 *__restrict__ base,
+                                          int ld, int nv, int gl, unsigned gmask,
+                                          float (&acc)[NCH][ElemTraits<T>::kVec]) {
+  for (int b = 0; b < len; b += G) {
+    const int cnt = min(G, len - b);
+    const int myc = __ldg(colp + b + min(gl, cnt - 1));
+    int t = 0;
+    for (; t + UNR <= cnt; t += UNR) {
+      uint4 v[UNR][NCH];
+#pragma unroll
+      for (int u = 0; u < UNR; ++u) {
+        const uint4 *src = base + (int64_t)__shfl_sync(gmask, myc, t + u, G) * ld;
+#pragma unroll
+        for (int i = 0; i < NCH; ++i)
+          v[u][i] = (FULL || gl + i * G < nv) ? __ldg(src + i * G) : make_uint4(0u, 0u, 0u, 0u);
+      }
+#pragma unroll
+      for (int u = 0; u < UNR; ++u)
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) add_chunk(acc[i], v[u][i], T());
+    }
+    for (; t < cnt; ++t) {
+      const uint4 *src = base + (int64_t)__shfl_sync(gmask, myc, t, G) * ld;
+#pragma unroll
+      for (int i = 0; i < NCH; ++i)
+        if (FULL || gl + i * G < nv) add_chunk(acc[i], __ldg(src + i * G), T());
+    }
+  }
+}
+
+// the first nloc[r] entries of row r read rows of X, the others slot rows (base stored pre-offset by -n rows)
+struct SumSrc {
+  const uint4 *b0, *b1s;
+  int ld0, ld1;
+  const int32_t *nloc;
+  const float *row_scale;   // 1 / deg(r)
+};
+
+template <typename T, int NCH, bool FULL>
+__device__ __forceinline__ void store_scaled(float (&acc)[NCH][ElemTraits<T>::kVec], float s, T *__restrict__ O,
+                                             int64_t ldo, int r, int gl, int G, int nv) {
+  constexpr int V = ElemTraits<T>::kVec;
+  uint4 *dst = reinterpret_cast<uint4 *>(O + (int64_t)r * ldo);
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    const int ch = gl + i * G;
+    if (FULL || ch < nv) {
+#pragma unroll
+      for (int j = 0; j < V; ++j) acc[i][j] *= s;
+      dst[ch] = pack16(acc[i], T());
+    }
+  }
+}
+
+// residency of the sum kernels: eight gathers in flight per lane need 64 registers
+constexpr int sum_blocks_per_sm(int nch, int unr) { return nch == 1 ? (unr <= 4 ? 5 : 4) : 1; }
+
+template <typename T, int G, int NCH, int UNR, bool FULL>
+__global__ void __launch_bounds__(256, sum_blocks_per_sm(NCH, UNR))
+    spmm_sum_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col, const int32_t *__restrict__ rows,
+                    int count, SumSrc ss, T *__restrict__ O, int64_t ldo, int nv) {
+  constexpr int V = ElemTraits<T>::kVec;
+  const int task = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G);
+  const int gl = threadIdx.x % G;
+  if (task >= count) return;
+  const unsigned gmask = group_mask<G>();
+  const int r = __ldg(rows + task);
+  float acc[NCH][V];
+#pragma unroll
+  for (int i = 0; i < NCH; ++i)
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
+  const int64_t e0 = rp[r];
+  const int len = (int)(rp[r + 1] - e0);
+  const int nl = __ldg(ss.nloc + r);
+  sum_range<T, G, NCH, UNR, FULL>(col + e0, nl, ss.b0 + gl, ss.ld0, nv, gl, gmask, acc);
+  if (len > nl) sum_range<T, G, NCH, UNR, FULL>(col + e0 + nl, len - nl, ss.b1s + gl, ss.ld1, nv, gl, gmask, acc);
+  store_scaled<T, NCH, FULL>(acc, __ldg(ss.row_scale + r), O, ldo, r, gl, G, nv);
+}
+
+// Hubs: one CTA per row.  Every warp (and, for rows narrower than 512 bytes, every lane group of a warp) takes a
+// contiguous share of the local and of the halo entries; the partial sums meet by a fixed shuffle tree and
+// an ordered shared-memory reduction.
+template <typename T, int G, int NCH, int UNR, bool FULL>
+__global__ void __launch_bounds__(256, sum_blocks_per_sm(NCH, UNR))
+    spmm_sum_hub_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ col,
+                        const int32_t *__restrict__ rows, SumSrc ss, T *__restrict__ O, int64_t ldo, int nv) {
+  extern __shared__ float hub_part[];
+  constexpr int V = ElemTraits<T>::kVec;
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int nwarps = blockDim.x / 32;
+  const int r = __ldg(rows + blockIdx.x);
+  const int64_t e0 = rp[r];
+  const int len = (int)(rp[r + 1] - e0);
+  const int nl = __ldg(ss.nloc + r);
+  constexpr int kGroups = 32 / G;
+  const int gl = lane % G, gi = lane / G;
+  const unsigned gmask = group_mask<G>();
+  const int shares = nwarps * kGroups;
+  const int mine = warp * kGroups + gi;
+  float acc[NCH][V];
+#pragma unroll
+  for (int i = 0; i < NCH; ++i)
+#pragma unroll
+    for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
+  auto share = [&](int total, int &b0, int &b1) {
+    const int per = ((total + shares - 1) / shares + G - 1) / G * G;
+    b0 = min(total, mine * per);
+    b1 = min(total, b0 + per);
+  };
+  int b0, b1;
+  share(nl, b0, b1);
+  if (b1 > b0) sum_range<T, G, NCH, UNR, FULL>(col + e0 + b0, b1 - b0, ss.b0 + gl, ss.ld0, nv, gl, gmask, acc);
+  share(len - nl, b0, b1);
+  if (b1 > b0) sum_range<T, G, NCH, UNR, FULL>(col + e0 + nl + b0, b1 - b0, ss.b1s + gl, ss.ld1, nv, gl, gmask, acc);
+#pragma unroll
+  for (int off = G; off < 32; off <<= 1)
+#pragma unroll
+    for (int i = 0; i < NCH; ++i)
+#pragma unroll
+      for (int j = 0; j < V; ++j) acc[i][j] += __shfl_xor_sync(0xFFFFFFFFu, acc[i][j], off);
+  const int row_floats = nv * V;
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    const int c = gl + i * G;
+    if (gi == 0 && c < nv)
+#pragma unroll
+      for (int j = 0; j < V; ++j) hub_part[(size_t)warp * row_floats + c * V + j] = acc[i][j];
+  }
+  __syncthreads();
+  const float s = __ldg(ss.row_scale + r);
+  uint4 *dst = reinterpret_cast<uint4 *>(O + (int64_t)r * ldo);
+  for (int c = threadIdx.x; c < nv; c += blockDim.x) {
+    float f[V];
+#pragma unroll
+    for (int j = 0; j < V; ++j) f[j] = 0.f;
+    for (int w = 0; w < nwarps; ++w)
+#pragma unroll
+      for (int j = 0; j < V; ++j) f[j] += hub_part[(size_t)w * row_floats + c * V + j];
+#pragma unroll
+    for (int j = 0; j < V; ++j) f[j] *= s;
+    dst[c] = pack16(f, T());
+  }
+}
+
+struct SumArgs {
+  const int64_t *rp;
+  const int32_t *col;
+  RowClass hubs, normal, shorts;
+  SumSrc ss;
+  void *O;
+  int64_t ldo;
+  int nv;
+};
+
+// G lanes x NCH chunks for hub and ordinary rows; the few rows of at most 8 entries take GS lanes x NCHS chunks
+template <typename T, int G, int NCH, int UNR, int GS, int NCHS>
+int launch_sum(const SumArgs &a, cudaStream_t st) {
+  constexpr int V = ElemTraits<T>::kVec;
+  const int threads = 256;
+  if (a.hubs.count) {
+    constexpr int GH = G < 8 ? 8 : G, NH = G < 8 ? 1 : NCH;
+    const size_t row_bytes = (size_t)a.nv * V * sizeof(float);
+    int warps = 8;
+    while (warps > 1 && warps * row_bytes > 48 * 1024) warps /= 2;
+    if (a.nv == GH * NH)
+      spmm_sum_hub_kernel<T, GH, NH, UNR, true><<<a.hubs.count, warps * 32, warps * row_bytes, st>>>(
+          a.rp, a.col, a.hubs.rows, a.ss, (T *)a.O, a.ldo, a.nv);
+    else
+      spmm_sum_hub_kernel<T, GH, NH, UNR, false><<<a.hubs.count, warps * 32, warps * row_bytes, st>>>(
+          a.rp, a.col, a.hubs.rows, a.ss, (T *)a.O, a.ldo, a.nv);
+    VARCO_KERNEL_LAUNCHED();
+  }
+  if (a.normal.count) {
+    const unsigned grid = (unsigned)(((int64_t)a.normal.count * G + threads - 1) / threads);
+    if (a.nv == G * NCH)
+      spmm_sum_kernel<T, G, NCH, UNR, true><<<grid, threads, 0, st>>>(a.rp, a.col, a.normal.rows, a.normal.count, a.ss,
+                                                                     (T *)a.O, a.ldo, a.nv);
+    else
+      spmm_sum_kernel<T, G, NCH, UNR, false><<<grid, threads, 0, st>>>(a.rp, a.col, a.normal.rows, a.normal.count, a.ss,
+                                                                      (T *)a.O, a.ldo, a.nv);
+    VARCO_KERNEL_LAUNCHED();
+  }
+  if (a.shorts.count) {
+    const unsigned grid = (unsigned)(((int64_t)a.shorts.count * GS + threads - 1) / threads);
+    if (a.nv == GS * NCHS)
+      spmm_sum_kernel<T, GS, NCHS, 1, true><<<grid, threads, 0, st>>>(a.rp, a.col, a.shorts.rows, a.shorts.count, a.ss,
+                                                                     (T *)a.O, a.ldo, a.nv);
+    else
+      spmm_sum_kernel<T, GS, NCHS, 1, false><<<grid, threads, 0, st>>>(a.rp, a.col, a.shorts.rows, a.shorts.count, a.ss,
+                                                                      (T *)a.O, a.ldo, a.nv);
+    VARCO_KERNEL_LAUNCHED();
+  }
+  return VARCO_OK;
+}
+
+template <typename T>
+int dispatch_sum(const SumArgs &a, cudaStream_t st) {
+  const int w = a.nv;
+  if (w <= 4) return launch_sum<T, 4, 1, 4, 4, 1>(a, st);
+  if (w <= 8) return launch_sum<T, 8, 1, 4, 4, 2>(a, st);
+  if (w <= 16) return launch_sum<T, 16, 1, 8, 4, 4>(a, st);
+  if (w <= 32) return launch_sum<T, 32, 1, 8, 8, 4>(a, st);
+  if (w <= 64) return launch_sum<T, 32, 2, 4, 16, 4>(a, st);
+  if (w <= 96) return launch_sum<T, 32, 3, 2, 16, 6>(a, st);
+  if (w <= 128) return launch_sum<T, 32, 4, 2, 32, 4>(a, st);
+  if (w <= 256) return launch_sum<T, 32, 8, 1, 32, 8>(a, st);
   return VARCO_UNSUPPORTED;
 }
 
@@ -861,6 +1123,25 @@ int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, cons
   a.short_col = pl->d.short_f_col;
   a.short_val = pl->d.short_f_val;
   a.short_nlocal = (int)pl->short_f.size();
+  if (a.panels == 1 && !pl->row_scale.empty() && (ldx % V) == 0 && (ldh % V) == 0) {
+    // mean aggregation: unweighted sums, one scale per finished row
+    SumArgs u{};
+    u.rp = a.rp;
+    u.col = a.col;
+    u.hubs = a.hubs;
+    u.normal = a.normal;
+    u.shorts = a.shorts;
+    u.ss.b0 = reinterpret_cast<const uint4 *>(X);
+    u.ss.ld0 = (int)(ldx / V);
+    u.ss.ld1 = (int)(ldh / V);
+    u.ss.b1s = reinterpret_cast<const uint4 *>(Xhalo) - (int64_t)pl->n * u.ss.ld1;
+    u.ss.nloc = pl->d.nloc;
+    u.ss.row_scale = pl->d.row_scale;
+    u.O = Agg;
+    u.ldo = ldagg;
+    u.nv = nv;
+    return dt == VARCO_F32 ? dispatch_sum<float>(u, st) : dispatch_sum<__nv_bfloat16>(u, st);
+  }
   return dt == VARCO_F32 ? dispatch<float>(a, st) : dispatch<__nv_bfloat16>(a, st);
 }
 

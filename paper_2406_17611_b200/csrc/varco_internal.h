@@ -17,6 +17,8 @@ struct varco_dev_image {
   const int32_t *nloc = nullptr;   // leading entries of a forward row that point at local rows
   const int32_t *col = nullptr;
   const float *val = nullptr;
+  // mean aggregation only: 1 / deg(r), the one weight every entry of row r carries (0 for an isolated row)
+  const float *row_scale = nullptr;
   // transposed structure: source u (row or n + slot) is used by rows colT[e] with weight valT[e]
   const int64_t *rpT = nullptr;
   const int32_t *colT = nullptr;
@@ -61,7 +63,7 @@ struct varco_plan {
   std::vector<int32_t> order_f, order_t, hub_f, hub_t, short_f, short_t, nloc;
   std::vector<int32_t> order_f_start, order_t_start, hub_f_start, hub_t_start, short_f_start, short_t_start;
   std::vector<int64_t> rp, rpT;
-  std::vector<float> val, valT, short_f_val, short_t_val;
+  std::vector<float> val, valT, short_f_val, short_t_val, row_scale;
   std::vector<int32_t> short_f_col, short_t_col;
   // device image
   bool uploaded = false;
