@@ -108,6 +108,32 @@ class Oracle:
             raise ValueError("bad schedule arguments")
         return int(num.value), int(den.value)
 
+    def schedule_fixed_increment(self, epoch, r0, R, den):
+        """Ratio (num, den) of the fixed-increment rate schedule r_{k+1} = r_k + R/den, r_0 = r0/den."""
+        num, d = C.c_uint64(), C.c_uint64()
+        rc = self.lib.orc_schedule_fixed_increment(epoch, C.c_uint64(r0), C.c_uint64(R), C.c_uint64(den),
+                                                   C.byref(num), C.byref(d))
+        if rc != 0:
+            raise ValueError("bad schedule arguments")
+        return int(num.value), int(d.value)
+
+    def schedule_rate_linear(self, epoch, r0, alpha, den):
+        """Ratio (num, den) of the linear rate schedule r_k = (alpha k + r0) / den, clipped at 1."""
+        num, d = C.c_uint64(), C.c_uint64()
+        rc = self.lib.orc_schedule_rate_linear(epoch, C.c_uint64(r0), C.c_uint64(alpha), C.c_uint64(den),
+                                               C.byref(num), C.byref(d))
+        if rc != 0:
+            raise ValueError("bad schedule arguments")
+        return int(num.value), int(d.value)
+
+    def schedule_exponential(self, epoch, K, beta):
+        """Ratio (num, 1) of the exponential rate schedule r_k = beta^-(K - k + 1), k = epoch + 1."""
+        num, d = C.c_uint64(), C.c_uint64()
+        rc = self.lib.orc_schedule_exponential(epoch, K, beta, C.byref(num), C.byref(d))
+        if rc != 0:
+            raise ValueError("bad schedule arguments")
+        return int(num.value), int(d.value)
+
     def set_threads(self, t):
         self.lib.orc_set_threads(t)
 

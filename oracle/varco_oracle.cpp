@@ -18,7 +18,9 @@
 //                                        through a shared key, zeros elsewhere
 //   * backward through the compressor -- Algorithm 1 (back-propagate across machines
 //                                        through the compression routine), Section III-A
-//   * scheduler                       -- Section IV and the appendix "Scheduler"
+//   * scheduler                       -- Section IV and the appendix "Scheduler" (linear ratio schedule
+//                                        of the experiments; fixed-increment, linear and exponential
+//                                        rate schedules; fixed ratios and "no communication" of Section V)
 //
 // All floating point is fp64.  Loops are written in the order of the
 // algorithm's steps; there is no blocking or fusion.  OpenMP is used only on
@@ -116,8 +118,12 @@ struct KeyedPerm {
 // ---------------------------------------------------------------- rate -> kept elements
 // Definition 1 sends F / c values; c is kept as the exact rational num/den.
 // Reading for non-integer F/c: k = ceil(F / c) clamped to [1, F].
+// den == 0 stands for the "no communication" setting of Section V (Tables II-III): an unbounded
+// ratio, nothing is sent, k = 0, and every remote row is the all-zero vector at the receiver.
 int kept_elements(int F, uint64_t num, uint64_t den) {
-  if (F <= 0 || num == 0 || den == 0 || num < den) return -1;
+  if (F <= 0 || num == 0) return -1;
+  if (den == 0) return 0;
+  if (num < den) return -1;
   uint64_t k = ((uint64_t)F * den + num - 1) / num;
   if (k < 1) k = 1;
   if (k > (uint64_t)F) k = (uint64_t)F;
@@ -324,6 +330,54 @@ int orc_schedule_linear(int epoch, int K, int a, int c_max, int c_min, uint64_t*
   if (v < (int64_t)c_min * K) v = (int64_t)c_min * K;
   *num = (uint64_t)v;
   *den = (uint64_t)K;
+  return 0;
+}
+
+// The other schedulers of the appendix "Scheduler".  There r_k is the communicated FRACTION (the
+// "compress rate", increasing while training); the ratio handed to the compressor is c_k = 1 / r_k.
+// Fractions are kept as integers over a common denominator, clipped at 1 (full communication).
+//
+// Fixed increment, written as the recurrence it is stated as: r_0 = r0/den, r_{k+1} = r_k + R/den.
+int orc_schedule_fixed_increment(int epoch, uint64_t r0, uint64_t R, uint64_t den, uint64_t* num_out,
+                                 uint64_t* den_out) {
+  if (epoch < 0 || den == 0 || r0 == 0 || r0 > den) return -1;
+  uint64_t r = r0;
+  for (int e = 0; e < epoch; ++e) {
+    r += R;
+    if (r > den) r = den;
+  }
+  *num_out = den;   // c = 1 / (r / den) = den / r
+  *den_out = r;
+  return 0;
+}
+// Linear increase in closed form: r_k = alpha k + r_0 with alpha = alpha_num/den, r_0 = r0/den.
+int orc_schedule_rate_linear(int epoch, uint64_t r0, uint64_t alpha_num, uint64_t den, uint64_t* num_out,
+                             uint64_t* den_out) {
+  if (epoch < 0 || den == 0 || r0 == 0 || r0 > den) return -1;
+  // alpha k + r_0 >= 1 as soon as k >= (den - r0) / alpha_num: clip there without forming the product
+  uint64_t r = den;
+  if (alpha_num == 0) r = r0;
+  else if ((uint64_t)epoch <= (den - r0) / alpha_num) r = r0 + alpha_num * (uint64_t)epoch;
+  if (r > den) r = den;
+  *num_out = den;
+  *den_out = r;
+  return 0;
+}
+// Exponential increase r_k = 1 / beta^(K - k + 1), k = 1..K; epoch e = k - 1, so c_e = beta^(K - e):
+// the last epoch e = K - 1 still compresses by beta (full communication would be step K + 1).
+// The power saturates at 2^32 - 1 (any ratio above the row width keeps one element).
+int orc_schedule_exponential(int epoch, int K, int beta, uint64_t* num_out, uint64_t* den_out) {
+  if (epoch < 0 || K < 1 || beta < 2) return -1;
+  uint64_t c = 1;
+  for (int i = 0; i < K - epoch; ++i) {
+    c *= (uint64_t)beta;
+    if (c > 0xFFFFFFFFull) {
+      c = 0xFFFFFFFFull;
+      break;
+    }
+  }
+  *num_out = c;
+  *den_out = 1;
   return 0;
 }
 
