@@ -219,6 +219,25 @@ class Workload:
         return w_self, w_neigh, bias
 
 
+def planted_task(block: np.ndarray, width: int, seed: int, signal: float = 0.12, train_share: float = 0.5):
+    """A node-classification task that needs the neighbours: features are N(0,1) noise plus a faint shift
+    signal * mu_b shared by the nodes of community b (about one standard deviation per node along mu_b, so that
+    a node's own row says little and the mean over its mostly same-community neighbours says a lot), two classes
+    per community: class = 2 * community + 1[x . v > 0] for one fixed direction v (the part a node can read off
+    its own row).  Returns (X fp32 [n x width], labels int64 [n], train mask bool [n]); draws inputs only."""
+    rng = np.random.default_rng(seed)
+    n = block.shape[0]
+    nb = int(block.max()) + 1
+    mu = rng.standard_normal((nb, width)).astype(np.float32)
+    v = rng.standard_normal(width).astype(np.float32)
+    x = rng.standard_normal((n, width), dtype=np.float32)
+    x += signal * mu[block]
+    coin = (x @ v > 0).astype(np.int64)
+    labels = 2 * block.astype(np.int64) + coin
+    train = rng.random(n) < train_share
+    return x, labels, train
+
+
 def make_workload(name: str, scale: float = 1.0, seed: int = 2406) -> Workload:
     """Build one of the named configurations.
 
@@ -229,6 +248,8 @@ def make_workload(name: str, scale: float = 1.0, seed: int = 2406) -> Workload:
          SAGE 100-256-256-47, bf16
     c4   Chung-Lu lognormal (mean degree 490), 233,000 nodes, random 8-way split, GCN 602-256-41, bf16
     c5   the c3 graph with a 4-layer SAGE 100-256-256-256-47, bf16
+    arx  citation-network shape: 169,343 nodes, ~1.16M undirected edges, 128-d, 40 classes, SAGE 128-256-256-40,
+         bf16, 16 random parts (arxiv_shaped() takes the number of parts and the kind of split)
 
     `scale` < 1 shrinks the node count (same degree law) for tests.
     """
@@ -262,4 +283,24 @@ def make_workload(name: str, scale: float = 1.0, seed: int = 2406) -> Workload:
         part = partition_random_equal(n, 8, seed + 1)
         return Workload("c4", rp, col, part, 8, "gcn", [602, 256, 41], True, 41, seed,
                         "Chung-Lu lognormal n=%d mean degree %.0f, random 8-way split" % (n, mean_deg))
+    if key == "arx":
+        return arxiv_shaped(16, "random", scale, seed)
     raise ValueError("unknown workload %r" % name)
+
+
+def arxiv_shaped(parts: int = 16, split: str = "random", scale: float = 1.0, seed: int = 2406) -> Workload:
+    """A citation-network-shaped second workload: 169,343 nodes, about 1.16M undirected edges (power-law degrees,
+    exponent 2.4), 128-d features, 40 classes, 3-layer SAGE 128-256-256-40, bf16; `parts` in {2, 4, 8, 16} equal
+    partitions, either a random split or contiguous ranges of a breadth-first order (the low-cut stand-in for a
+    partitioner).  The small-graph regime: a few MB per layer, where launches and tiny segments dominate."""
+    n = max(1000, int(round(169343 * scale)))
+    m = int(round(1166243 * scale))
+    rp, col = chung_lu_power_law(n, m, 2.4, seed + 3)
+    if split == "random":
+        part = partition_random_equal(n, parts, seed + 1)
+    elif split == "bfs":
+        part = partition_bfs_ranges(rp, col, parts, seed + 1)
+    else:
+        raise ValueError("split must be 'random' or 'bfs'")
+    return Workload("arx", rp, col, part, parts, "sage", [128, 256, 256, 40], True, 40, seed,
+                    "Chung-Lu power law n=%d (citation-network shape), %d %s equal parts" % (n, parts, split))

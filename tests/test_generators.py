@@ -72,3 +72,25 @@ def test_generators_are_deterministic():
     x = a.features()
     assert np.array_equal(synth.bf16_round(x), x)             # already bf16-representable
     assert abs(float(x.std()) - 1.0) < 0.02
+
+
+def test_citation_shaped_workload_and_its_partition_sweep(orc):
+    """The second workload (citation-network shape: 169,343 nodes, ~1.16M undirected edges, 128-d, 40 classes)
+    over Q in {2, 4, 8, 16} workers: a random equal split leaves 1 - 1/Q of the entries across workers (the
+    arithmetic of Table I's random rows), ranges of a breadth-first order cut fewer."""
+    _, size = _table1()
+    nodes, edges = size["arxiv"]
+    full = synth.arxiv_shaped(16, "random")
+    assert full.n == nodes and full.widths == [128, 256, 256, 40] and full.classes == 40
+    assert abs(full.nnz / 2 - edges) / edges < 0.02          # duplicates dropped: within 2 % of the edge count
+    for Q in (2, 4, 8, 16):
+        shares = {}
+        for split in ("random", "bfs"):
+            wl = synth.arxiv_shaped(Q, split, scale=0.1)
+            sizes = np.bincount(wl.part, minlength=Q)
+            assert wl.parts == Q and sizes.max() - sizes.min() <= 1
+            g = orc.graph(wl.row_ptr, wl.col, wl.part, Q, "sage")
+            assert g.cross_entries + g.self_entries == wl.nnz
+            shares[split] = g.cross_entries / wl.nnz
+        assert abs(shares["random"] - (1 - 1 / Q)) < 0.02
+        assert shares["bfs"] < shares["random"]
