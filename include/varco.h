@@ -67,8 +67,8 @@ typedef struct { uint64_t seed; uint32_t epoch, layer; } varco_key_t;
 const char *varco_status_string(int status);
 
 /* ------------------------------------------------------------------------------------------
- * Plan: partition and halo structure (Section III, "each machine is equipped with a subset of
- * the graph"; the boundary nodes of Section III are the halo rows).
+ * Plan: partition and halo structure (Section III: every worker holds the nodes of one partition;
+ * the boundary nodes of that section are the halo rows).
  *
  * varco_partition_build
  *   n, row_ptr[n+1], col_idx[nnz]  host CSR adjacency: row i lists the nodes j that i aggregates
@@ -84,8 +84,11 @@ const char *varco_status_string(int status);
  *   (rows it receives) by (owner partition p ascending, original id ascending); the send segments
  *   of partition p by (destination q ascending, original id ascending).
  *   halo(p->q) = { j owned by p : some i owned by q has an entry (i, j) }, p != q.
- *   Errors: INVALID_ARG, BAD_GRAPH, BAD_PARTITION, NOMEM, UNSUPPORTED (n or nnz + n + H_total
- *   beyond 2^31 - 1).
+ *   Errors: INVALID_ARG, BAD_GRAPH, BAD_PARTITION, NOMEM, UNSUPPORTED (n or n + H_total beyond
+ *   2^31 - 1: rows and halo slots share one 32-bit index space; the number of stored entries is
+ *   not limited, entry offsets are 64-bit).
+ *   Inputs of the layer entry points must be finite: the weighted aggregation kernels pad their
+ *   gather batches with zero-weight copies of a real source row, and 0 * Inf is NaN.
  */
 int varco_partition_build(int64_t n, const int64_t *row_ptr, const int32_t *col_idx,
                           const int32_t *part, int32_t P, varco_conv_t conv, varco_plan_t **out);
@@ -148,6 +151,22 @@ int varco_workspace_bytes(const varco_plan_t *plan, int32_t F_in_max, int32_t F_
 int varco_kept(int32_t F, varco_ratio_t c, int32_t *k);
 int varco_schedule_linear(int32_t epoch, int32_t K, int32_t slope_a, int32_t c_max, int32_t c_min,
                           varco_ratio_t *c);
+
+/* The other schedulers of the appendix "Scheduler".  There r_k is the communicated fraction ("compress rate",
+ * raised while training) and the compressor is handed c_k = 1 / r_k.
+ *   varco_schedule_rate_linear   r_k = (alpha k + r0) / den clipped at 1 (full communication); the fixed
+ *                                increment r_{k+1} = r_k + R of the same appendix is this sequence with
+ *                                alpha = R.  Returns c = den / (alpha k + r0) as the exact rational.
+ *                                INVALID_ARG unless 0 < r0 <= den and epoch >= 0.
+ *   varco_schedule_exponential   r_k = 1 / beta^(K - k + 1) for steps k = 1..K, epoch = k - 1, i.e.
+ *                                c = beta^(K - epoch) (the last epoch still compresses by beta; epochs >= K
+ *                                give 1); the power saturates at 2^32 - 1.  INVALID_ARG unless beta >= 2,
+ *                                K >= 1, epoch >= 0.
+ * The fixed ratios of Section V are the constant {c, 1}; its "no communication" setting is a ratio with
+ * den = 0: varco_kept returns k = 0 for it, the layer entry points then send nothing (halo_bytes = 0) and
+ * every remote neighbour contributes the zero vector, forward and backward. */
+int varco_schedule_rate_linear(int32_t epoch, uint32_t r0, uint32_t alpha, uint32_t den, varco_ratio_t *c);
+int varco_schedule_exponential(int32_t epoch, int32_t K, int32_t beta, varco_ratio_t *c);
 
 /* ------------------------------------------------------------------------------------------
  * Compression over all halo copies of the plan (Algorithm 1, second step; Definition 1;
@@ -284,6 +303,26 @@ int varco_profile_read(varco_plan_t *plan, int64_t *launches /* [VARCO_STAGE_COU
  * `milliseconds`, `count` receives how many exist.  Synchronises the events it reads. */
 int varco_profile_spans(varco_plan_t *plan, int32_t stage, double *milliseconds, int64_t capacity,
                         int64_t *count);
+/* Debug build (no counterpart in the paper).  A library compiled with -DVARCO_DEBUG checks, on the device,
+ * every source row, destination row and kept position its aggregation kernels index against the extent of the
+ * array it addresses; a failed check records a code (11 source row, 12 destination row, 13 kept position) and
+ * skips the access -- nothing traps.  The same build validates the plan's index arrays on the host at upload
+ * (BAD_GRAPH), puts 256 guard bytes behind every workspace segment, and reports a damaged guard block as bit 30
+ * of varco_workspace_status.  This call synchronises the device and returns the first recorded code (0 = none)
+ * and clears it; in a release build is_debug_build = 0 and word = 0. */
+int varco_debug_status(int32_t *is_debug_build, int32_t *word);
+/* Random-row gather probe (no counterpart in the paper; a measurement aid).  Every output row is the
+ * bitwise XOR of `per_out` rows of `table`, picked by `index`; nothing else is computed, so the time of the
+ * launch is the time the memory system needs for out_rows * per_out random row reads.  The benchmark calls
+ * it on a table that fits L2 and on one that does not: those two rates are what the aggregation stages,
+ * which read one feature row per stored entry, are measured against.
+ *   table  device, [table_rows x row_chunks * 16 bytes], 16-byte aligned; row_chunks in {8, 16, 32}
+ *   index  device int32 [out_rows x per_out], 16-byte aligned, per_out a positive multiple of 4; values are
+ *          clamped into [0, table_rows) by the kernel
+ *   out    device, [out_rows x row_chunks * 16 bytes]
+ * Enqueued on `stream`, no synchronisation.  INVALID_ARG / UNSUPPORTED on anything else. */
+int varco_probe_gather(const void *table, int64_t table_rows, int32_t row_chunks, const int32_t *index,
+                       int64_t out_rows, int32_t per_out, void *out, void *stream);
 /* Number of CUDA kernels this library has launched in this process so far (all plans, all
  * streams).  Also a measurement aid without a counterpart in the paper. */
 int varco_kernel_launches(int64_t *count);

@@ -22,8 +22,9 @@ STAGES = ["compress", "decompress", "spmm", "gemm_fwd", "gemm_dx", "gemm_dw", "s
 EXPORTS = ["varco_status_string", "varco_partition_build", "varco_partition_destroy", "varco_partition_info",
            "varco_partition_boundary_rows", "varco_partition_set_l2_budget", "varco_partition_gather_model", "varco_partition_counts", "varco_partition_halo", "varco_partition_perm", "varco_partition_device_bytes",
            "varco_partition_upload", "varco_workspace_bytes", "varco_kept", "varco_schedule_linear",
+           "varco_schedule_rate_linear", "varco_schedule_exponential",
            "varco_compress", "varco_decompress", "varco_layer_fwd", "varco_layer_bwd", "varco_profile_enable",
-           "varco_profile_reset", "varco_profile_read", "varco_profile_spans", "varco_kernel_launches", "varco_workspace_status",
+           "varco_profile_reset", "varco_profile_read", "varco_profile_spans", "varco_probe_gather", "varco_debug_status", "varco_kernel_launches", "varco_workspace_status",
            "varco_exchange_noalloc"]
 
 
@@ -54,10 +55,11 @@ def lib():
     global _lib
     if _lib is not None:
         return _lib
-    if not os.path.exists(LIB_PATH):
-        raise ImportError("libvarco.so is not built: run `python -m paper_2406_17611_b200.build` "
-                          "(there is no CPU fallback)")
-    L = C.CDLL(LIB_PATH)
+    path = os.environ.get("VARCO_LIBRARY", LIB_PATH)    # e.g. the debug build, libvarco_debug.so
+    if not os.path.exists(path):
+        raise ImportError("%s is not built: run `python -m paper_2406_17611_b200.build` "
+                          "(there is no CPU fallback)" % os.path.basename(path))
+    L = C.CDLL(path)
     vp, i64p, i32p = C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int32)
     L.varco_status_string.restype = C.c_char_p
     L.varco_status_string.argtypes = [C.c_int]
@@ -75,6 +77,8 @@ def lib():
     L.varco_workspace_bytes.argtypes = [vp, C.c_int32, C.c_int32, C.c_int, C.POINTER(C.c_size_t)]
     L.varco_kept.argtypes = [C.c_int32, Ratio, i32p]
     L.varco_schedule_linear.argtypes = [C.c_int32] * 5 + [C.POINTER(Ratio)]
+    L.varco_schedule_rate_linear.argtypes = [C.c_int32, C.c_uint32, C.c_uint32, C.c_uint32, C.POINTER(Ratio)]
+    L.varco_schedule_exponential.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.POINTER(Ratio)]
     L.varco_compress.argtypes = [vp, vp, C.c_int64, C.c_int32, C.c_int, Ratio, Key, vp, C.POINTER(C.c_uint64), vp]
     L.varco_decompress.argtypes = [vp, vp, C.c_int32, C.c_int, Ratio, Key, vp, C.c_int64, vp]
     L.varco_exchange_noalloc.argtypes = [vp, vp, C.c_int64, C.c_int32, C.c_int, Ratio, Key, vp, C.c_int64,
@@ -87,6 +91,8 @@ def lib():
     L.varco_profile_reset.argtypes = [vp]
     L.varco_profile_read.argtypes = [vp, i64p, C.POINTER(C.c_double)]
     L.varco_profile_spans.argtypes = [vp, C.c_int32, C.POINTER(C.c_double), C.c_int64, i64p]
+    L.varco_probe_gather.argtypes = [vp, C.c_int64, C.c_int32, vp, C.c_int64, C.c_int32, vp, vp]
+    L.varco_debug_status.argtypes = [i32p, i32p]
     L.varco_kernel_launches.argtypes = [i64p]
     L.varco_workspace_status.argtypes = [vp, vp, i32p]
     _lib = L
@@ -127,6 +133,39 @@ def varco_schedule_linear(epoch, K, slope_a=5, c_max=128, c_min=1):
     _check(lib().varco_schedule_linear(int(epoch), int(K), int(slope_a), int(c_max), int(c_min), C.byref(r)),
            "varco_schedule_linear")
     return (int(r.num), int(r.den))
+
+
+NO_COMMUNICATION = (1, 0)   # ratio with denominator 0: nothing is sent (k = 0)
+
+
+def varco_schedule_rate_linear(epoch, r0, alpha, den):
+    """Ratio of the rate schedule r_k = (alpha k + r0) / den (also the fixed increment r_{k+1} = r_k + alpha/den)."""
+    r = Ratio()
+    _check(lib().varco_schedule_rate_linear(int(epoch), int(r0), int(alpha), int(den), C.byref(r)),
+           "varco_schedule_rate_linear")
+    return (int(r.num), int(r.den))
+
+
+def varco_schedule_exponential(epoch, K, beta):
+    """Ratio beta^(K - epoch) of the exponential rate schedule r_k = beta^-(K - k + 1), k = epoch + 1."""
+    r = Ratio()
+    _check(lib().varco_schedule_exponential(int(epoch), int(K), int(beta), C.byref(r)), "varco_schedule_exponential")
+    return (int(r.num), int(r.den))
+
+
+def varco_debug_status():
+    """(is this a -DVARCO_DEBUG build, first failed device-side index check since the last call or 0)."""
+    dbg, word = C.c_int32(), C.c_int32()
+    _check(lib().varco_debug_status(C.byref(dbg), C.byref(word)), "varco_debug_status")
+    return bool(dbg.value), int(word.value)
+
+
+def varco_probe_gather(table, index, out):
+    """Enqueue the random-row gather probe: out[r] = XOR of table[index[r, :]] (device tensors; rows of 128, 256
+    or 512 bytes)."""
+    row_bytes = table.stride(0) * table.element_size()
+    _check(lib().varco_probe_gather(_ptr(table), table.shape[0], row_bytes // 16, _ptr(index), index.shape[0],
+                                    index.shape[1], _ptr(out), _stream()), "varco_probe_gather")
 
 
 def varco_kernel_launches():
@@ -189,6 +228,10 @@ class Plan:
         _check(lib().varco_partition_gather_model(self.h, int(bool(transposed)), int(resident_rows), C.byref(e),
                                                   C.byref(s), C.byref(r)), "varco_partition_gather_model")
         return int(e.value), int(s.value), int(r.value)
+
+    def rows_per_partition(self):
+        """Number of rows of every partition (the plan's row order is partition-contiguous)."""
+        return np.bincount(self.part, minlength=self.P).astype(np.int64)
 
     def counts(self):
         out = np.zeros((self.P, self.P), dtype=np.int64)

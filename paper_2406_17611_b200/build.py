@@ -28,10 +28,17 @@ def _stale(target, deps):
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) -> str:
-    """Compile every source under csrc/ and link the shared library.  Returns its path."""
+def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False, debug: bool = False) -> str:
+    """Compile every source under csrc/ and link the shared library.  Returns its path.
+    debug=True builds libvarco_debug.so (-DVARCO_DEBUG: device-side index checks, workspace guard blocks) next
+    to the release library, from its own object folder."""
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    extra = os.environ.get("VARCO_NVCC_FLAGS", "").split()   # e.g. -DVARCO_DEBUG
+    extra = os.environ.get("VARCO_NVCC_FLAGS", "").split()
+    LIB, OBJ = globals()["LIB"], globals()["OBJ"]
+    if debug:
+        extra = extra + ["-DVARCO_DEBUG"]
+        LIB = os.path.join(HERE, "libvarco_debug.so")
+        OBJ = os.path.join(HERE, "_build", "debug")
     os.makedirs(OBJ, exist_ok=True)
     headers = glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh")) + \
         glob.glob(os.path.join(ROOT, "include", "*.h"))
@@ -63,4 +70,5 @@ def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) 
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, ptxas_info="--ptxas" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, ptxas_info="--ptxas" in sys.argv,
+                debug="--debug" in sys.argv))

@@ -23,6 +23,37 @@ void varco_count_launch();
   } while (0)
 
 // ------------------------------------------------------------------------------------------
+// Debug build (-DVARCO_DEBUG): every index a kernel gathers from or scatters to is checked against the extent
+// of the array it addresses.  A failed check records a code in the translation unit's debug word and the access
+// is skipped; nothing traps, the context stays usable.  varco_debug_status() collects the words.
+// Codes: 11 source row, 12 destination row, 13 kept position of the aggregation kernels.  The index arrays the
+// halo kernels walk are fixed at plan build time; the debug build validates them on the host when the plan is
+// uploaded (varco_partition_upload returns BAD_GRAPH on a damaged image).
+#ifdef VARCO_DEBUG
+#ifdef __CUDACC__
+static __device__ int varco_dbg_word;
+__device__ __forceinline__ bool varco_dbg_ok(long long idx, long long limit, int code) {
+  if (idx >= 0 && idx < limit) return true;
+  atomicCAS(&varco_dbg_word, 0, code);
+  return false;
+}
+// host side of one translation unit: read and clear its word
+#define VARCO_DEFINE_DEBUG_READER(name)                                              \
+  int name() {                                                                        \
+    int v = 0, zero = 0;                                                              \
+    if (cudaMemcpyFromSymbol(&v, varco_dbg_word, sizeof(int)) != cudaSuccess) return -1; \
+    cudaMemcpyToSymbol(varco_dbg_word, &zero, sizeof(int));                           \
+    return v;                                                                         \
+  }
+#endif
+#define VARCO_DBG_OK(idx, limit, code) varco_dbg_ok((long long)(idx), (long long)(limit), (code))
+#else
+#define VARCO_DBG_OK(idx, limit, code) (true)
+#define VARCO_DEFINE_DEBUG_READER(name) \
+  int name() { return 0; }
+#endif
+
+// ------------------------------------------------------------------------------------------
 // Shared-key permutation of [0, F): which positions of a row are sent (appendix "Compression
 // Mechanism": chosen at random at the encoder, known to the decoder through a shared key).
 // A 6-round balanced Feistel network over the smallest even-bit domain covering [0, F),

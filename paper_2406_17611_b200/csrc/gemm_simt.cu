@@ -4,7 +4,22 @@
 // Y = rho(Agg W + b) (GCN), and the matching backward products dZ W^T and [X | Agg]^T dZ.
 // This path serves the fp32 configurations, whose 1e-5 tolerance rules out bf16 / tf32 tensor
 // core inputs; the bf16 configurations use the tcgen05 kernels instead.
+#include <algorithm>
+#include <type_traits>
+
 #include "device_common.cuh"
+
+// SM count of the current device (sizes the split reductions)
+static int simt_sms() {
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+      sms = 148;   // no device visible (a build host): the part this library targets
+  }
+  return sms;
+}
 
 namespace {
 
@@ -112,6 +127,141 @@ __global__ void __launch_bounds__(256) gemm_kernel(int M, int N, Operand<T> p0, 
   }
 }
 
+// fp32 products of the fp32 configurations: 128 x 64 x 16 tiles, 8 x 4 outputs per thread, 16-byte global loads
+// and shared-memory reads, the next tile fetched into registers while the current one is multiplied (two
+// shared-memory buffers, one barrier per step).  Same contract as gemm_kernel<float, float, A_T, B_T>.
+constexpr int SM = 128, SN = 64, SK = 16;
+
+__device__ __forceinline__ float4 ld4(const float *p, bool vec, int valid) {
+  // 4 consecutive floats of which the first `valid` exist; one 16-byte load when the address allows it
+  if (vec && valid >= 4) return __ldg(reinterpret_cast<const float4 *>(p));
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (valid > 0) v.x = __ldg(p);
+  if (valid > 1) v.y = __ldg(p + 1);
+  if (valid > 2) v.z = __ldg(p + 2);
+  if (valid > 3) v.w = __ldg(p + 3);
+  return v;
+}
+
+template <bool A_T, bool B_T>
+__global__ void __launch_bounds__(256, 2) sgemm_kernel(int M, int N, Operand<float> p0, Operand<float> p1, int npairs,
+                                                       const float *__restrict__ bias, int relu, float *__restrict__ C,
+                                                       int64_t ldc, int k_chunk) {
+  __shared__ __align__(16) float As[2][SK][SM + 4];
+  __shared__ __align__(16) float Bs[2][SK][SN + 4];
+  const int tid = threadIdx.x, tx = tid % 16, ty = tid / 16;
+  const int m0 = blockIdx.x * SM, n0 = blockIdx.y * SN;
+  float acc[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (int pi = 0; pi < npairs; ++pi) {
+    const Operand<float> p = pi == 0 ? p0 : p1;
+    int kb = 0, ke = p.K;
+    if (A_T) {
+      kb = blockIdx.z * k_chunk;
+      ke = min(p.K, kb + k_chunk);
+    }
+    if (ke <= kb) continue;
+    const bool avec = (reinterpret_cast<uintptr_t>(p.A) & 15u) == 0 && (p.lda & 3) == 0 && (A_T || (kb & 3) == 0);
+    const bool bvec = (reinterpret_cast<uintptr_t>(p.B) & 15u) == 0 && (p.ldb & 3) == 0 && (!B_T || (kb & 3) == 0);
+    float4 ra[2], rb;
+    auto fetch = [&](int k0) {
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int idx = tid + i * 256;
+        if (A_T) {   // A is [K x M]: 16 rows of 128 consecutive outputs
+          const int kk = idx / 32, m = m0 + (idx % 32) * 4;
+          const int gk = k0 + kk;
+          ra[i] = (gk < ke) ? ld4(p.A + (int64_t)gk * p.lda + m, avec, M - m) : make_float4(0.f, 0.f, 0.f, 0.f);
+        } else {     // A is [M x K]: 128 rows of 16 consecutive k
+          const int m = m0 + idx / 4, gk = k0 + (idx % 4) * 4;
+          ra[i] = (m < M) ? ld4(p.A + (int64_t)m * p.lda + gk, avec, ke - gk) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+      if (B_T) {     // B is [N x K]: 64 rows of 16 consecutive k
+        const int nn = n0 + tid / 4, gk = k0 + (tid % 4) * 4;
+        rb = (nn < N) ? ld4(p.B + (int64_t)nn * p.ldb + gk, bvec, ke - gk) : make_float4(0.f, 0.f, 0.f, 0.f);
+      } else {       // B is [K x N]: 16 rows of 64 consecutive outputs
+        const int gk = k0 + tid / 16, nn = n0 + (tid % 16) * 4;
+        rb = (gk < ke) ? ld4(p.B + (int64_t)gk * p.ldb + nn, bvec, N - nn) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    };
+    auto stash = [&](int buf) {
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int idx = tid + i * 256;
+        if (A_T) {
+          *reinterpret_cast<float4 *>(&As[buf][idx / 32][(idx % 32) * 4]) = ra[i];
+        } else {
+          const int m = idx / 4, kk = (idx % 4) * 4;
+          As[buf][kk][m] = ra[i].x;
+          As[buf][kk + 1][m] = ra[i].y;
+          As[buf][kk + 2][m] = ra[i].z;
+          As[buf][kk + 3][m] = ra[i].w;
+        }
+      }
+      if (B_T) {
+        const int nn = tid / 4, kk = (tid % 4) * 4;
+        Bs[buf][kk][nn] = rb.x;
+        Bs[buf][kk + 1][nn] = rb.y;
+        Bs[buf][kk + 2][nn] = rb.z;
+        Bs[buf][kk + 3][nn] = rb.w;
+      } else {
+        *reinterpret_cast<float4 *>(&Bs[buf][tid / 16][(tid % 16) * 4]) = rb;
+      }
+    };
+    const int steps = (ke - kb + SK - 1) / SK;
+    __syncthreads();          // the buffers of the previous operand pair are no longer read
+    fetch(kb);
+    stash(0);
+    __syncthreads();
+    for (int s = 0; s < steps; ++s) {
+      const int buf = s & 1;
+      if (s + 1 < steps) fetch(kb + (s + 1) * SK);
+#pragma unroll
+      for (int kk = 0; kk < SK; ++kk) {
+        const float4 a0 = *reinterpret_cast<const float4 *>(&As[buf][kk][ty * 8]);
+        const float4 a1 = *reinterpret_cast<const float4 *>(&As[buf][kk][ty * 8 + 4]);
+        const float4 b = *reinterpret_cast<const float4 *>(&Bs[buf][kk][tx * 4]);
+        const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+        const float bb[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
+      }
+      if (s + 1 < steps) stash(buf ^ 1);
+      __syncthreads();
+    }
+  }
+  float *Cz = C;
+  if (A_T) Cz += (int64_t)blockIdx.z * M * ldc;
+  const int gn = n0 + tx * 4;
+  const bool cvec = (reinterpret_cast<uintptr_t>(Cz) & 15u) == 0 && (ldc & 3) == 0 && gn + 3 < N;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int gm = m0 + ty * 8 + i;
+    if (gm >= M) continue;
+    float v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      v[j] = acc[i][j];
+      if (bias && gn + j < N) v[j] += bias[gn + j];
+      if (relu) v[j] = fmaxf(v[j], 0.f);
+    }
+    if (cvec) {
+      *reinterpret_cast<float4 *>(Cz + (int64_t)gm * ldc + gn) = make_float4(v[0], v[1], v[2], v[3]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (gn + j < N) Cz[(int64_t)gm * ldc + gn + j] = v[j];
+    }
+  }
+}
+
 // out[i] = sum_z partial[z * count + i], z ascending (deterministic)
 __global__ void reduce_partials_kernel(const float *__restrict__ partial, int64_t count, int splits,
                                        float *__restrict__ out) {
@@ -203,18 +353,28 @@ __global__ void relu_mask_kernel(const T *__restrict__ Y, int64_t ldy, const T *
 template <typename T>
 int fwd_t(int n, int F_in, int F_out, const T *X, int64_t ldx, const T *Agg, int64_t lda, const T *Ws, const T *Wn,
           const float *bias, int relu, T *Y, int64_t ldy, cudaStream_t st) {
-  dim3 grid((n + BM - 1) / BM, (F_out + BN - 1) / BN, 1);
   Operand<T> pa{Agg, lda, Wn, F_out, F_in}, px{X, ldx, Ws, F_out, F_in};
-  gemm_kernel<T, T, false, false><<<grid, 256, 0, st>>>(n, F_out, pa, px, Ws ? 2 : 1, bias, relu, Y, ldy, 0);
+  if constexpr (std::is_same<T, float>::value) {
+    dim3 grid((n + SM - 1) / SM, (F_out + SN - 1) / SN, 1);
+    sgemm_kernel<false, false><<<grid, 256, 0, st>>>(n, F_out, pa, px, Ws ? 2 : 1, bias, relu, Y, ldy, 0);
+  } else {
+    dim3 grid((n + BM - 1) / BM, (F_out + BN - 1) / BN, 1);
+    gemm_kernel<T, T, false, false><<<grid, 256, 0, st>>>(n, F_out, pa, px, Ws ? 2 : 1, bias, relu, Y, ldy, 0);
+  }
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
 template <typename T>
 int dx_t(int n, int F_in, int F_out, const T *dZ, int64_t lddz, const T *W, T *out, int64_t ldo, cudaStream_t st) {
-  dim3 grid((n + BM - 1) / BM, (F_in + BN - 1) / BN, 1);
   Operand<T> p{dZ, lddz, W, F_out, F_out};
-  gemm_kernel<T, T, false, true><<<grid, 256, 0, st>>>(n, F_in, p, p, 1, nullptr, 0, out, ldo, 0);
+  if constexpr (std::is_same<T, float>::value) {
+    dim3 grid((n + SM - 1) / SM, (F_in + SN - 1) / SN, 1);
+    sgemm_kernel<false, true><<<grid, 256, 0, st>>>(n, F_in, p, p, 1, nullptr, 0, out, ldo, 0);
+  } else {
+    dim3 grid((n + BM - 1) / BM, (F_in + BN - 1) / BN, 1);
+    gemm_kernel<T, T, false, true><<<grid, 256, 0, st>>>(n, F_in, p, p, 1, nullptr, 0, out, ldo, 0);
+  }
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
@@ -222,12 +382,18 @@ int dx_t(int n, int F_in, int F_out, const T *dZ, int64_t lddz, const T *W, T *o
 }  // namespace
 
 // scratch floats needed by varco_simt_gemm_dw (split partials) and by varco_colsum
+// splits of the node range of a weight-gradient product: about two CTAs per SM over all tiles
+static int dw_splits(int tiles) {
+  int splits = (2 * simt_sms() + tiles - 1) / tiles;
+  return splits < 1 ? 1 : splits;
+}
+
 size_t varco_simt_dw_scratch_bytes(int F_in, int F_out) {
-  const int tiles = ((F_in + BM - 1) / BM) * ((F_out + BN - 1) / BN);
-  int splits = (2 * 148 + tiles - 1) / tiles;
-  if (splits < 1) splits = 1;
+  // the larger of the two tilings' split counts (fp32 tiles are 128 x 64, the generic ones 64 x 64)
+  const int t0 = ((F_in + BM - 1) / BM) * ((F_out + BN - 1) / BN), t1 = ((F_in + SM - 1) / SM) * ((F_out + SN - 1) / SN);
+  const int splits = std::max(dw_splits(t0), dw_splits(t1)) + 1;
   size_t a = (size_t)splits * (size_t)F_in * F_out * sizeof(float);
-  size_t b = (size_t)4 * 148 * F_out * sizeof(float);   // column-sum partials
+  size_t b = (size_t)4 * simt_sms() * F_out * sizeof(float);   // column-sum partials
   return (a > b ? a : b) + 256;
 }
 
@@ -255,14 +421,19 @@ int varco_simt_gemm_dx(int n, int F_in, int F_out, varco_dtype_t dt, const void 
 template <typename T>
 static int dw_t(int n, int F_in, int F_out, const T *A, int64_t lda, const T *dZ, int64_t lddz, float *dW,
                 float *scratch, cudaStream_t st) {
-  const int tiles = ((F_in + BM - 1) / BM) * ((F_out + BN - 1) / BN);
-  int splits = (2 * 148 + tiles - 1) / tiles;
+  constexpr bool f32 = std::is_same<T, float>::value;
+  const int tm = f32 ? SM : BM, tn = f32 ? SN : BN;
+  const int tiles = ((F_in + tm - 1) / tm) * ((F_out + tn - 1) / tn);
+  int splits = dw_splits(tiles);
   int chunk = (n + splits - 1) / splits;
   chunk = (chunk + BK - 1) / BK * BK;
   splits = (n + chunk - 1) / chunk;
-  dim3 grid((F_in + BM - 1) / BM, (F_out + BN - 1) / BN, splits);
+  dim3 grid((F_in + tm - 1) / tm, (F_out + tn - 1) / tn, splits);
   Operand<T> p{A, lda, dZ, lddz, n};
-  gemm_kernel<T, float, true, false><<<grid, 256, 0, st>>>(F_in, F_out, p, p, 1, nullptr, 0, scratch, F_out, chunk);
+  if constexpr (f32)
+    sgemm_kernel<true, false><<<grid, 256, 0, st>>>(F_in, F_out, p, p, 1, nullptr, 0, scratch, F_out, chunk);
+  else
+    gemm_kernel<T, float, true, false><<<grid, 256, 0, st>>>(F_in, F_out, p, p, 1, nullptr, 0, scratch, F_out, chunk);
   VARCO_KERNEL_LAUNCHED();
   const int64_t count = (int64_t)F_in * F_out;
   reduce_partials_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(scratch, count, splits, dW);
@@ -281,7 +452,7 @@ namespace {
 template <typename T>
 int colsum_t(int n, int F_out, const T *dZ, int64_t lddz, float *out, float *scratch, const T *Y, int64_t ldy,
              T *dZout, int64_t ldout, cudaStream_t st) {
-  int splits = 4 * 148;
+  int splits = 4 * simt_sms();
   int chunk = (n + splits - 1) / splits;
   if (chunk < 1) chunk = 1;
   splits = (n + chunk - 1) / chunk;

@@ -7,9 +7,10 @@
 //
 // Kernel 1 (rows_kernel): M = nodes.  A tiles [128 nodes x 64 features] are K-major straight from
 // the activation matrices; B tiles come from a repacked, zero-padded K-major copy of the weights.
-// One CTA per SM, persistent over (node tile, output tile) work items; warp 4 issues TMA, warp 5
-// issues tcgen05.mma into one of two TMEM accumulators, warps 0-3 drain the other accumulator
-// (tcgen05.ld), apply bias / ReLU, convert and store.
+// One CTA per SM, persistent over (node tile, output tile) work items; warp 8 issues the TMA loads,
+// warp 9 issues tcgen05.mma into one of two TMEM accumulators, warps 0-7 drain the other accumulator
+// (tcgen05.ld, two warps per TMEM lane quarter), apply bias / ReLU, convert, stage 64-column slabs in
+// swizzled shared-memory tiles and write them with TMA stores.
 //
 // Kernel 2 (dw_kernel): the reduction runs over nodes, so both operands are used MN-major: TMA
 // boxes of [64 nodes x 64 features] land in shared memory exactly as loaded from the row-major
@@ -569,7 +570,7 @@ int sm_count() {
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (sms <= 0) sms = 148;
+    if (sms <= 0) sms = 148;   // no device visible (a build host): the part this library targets
   }
   return sms;
 }
@@ -596,7 +597,7 @@ static size_t packed_bytes(int F_in, int F_out) {
   return (fwd + 255) / 256 * 256;
 }
 size_t varco_tc_scratch_bytes(int F_in, int F_out) {
-  const size_t partial = (size_t)148 * 2 * 128 * 256 * 4;           // groups x splits <= 148 CTAs, 2 tiles each
+  const size_t partial = (size_t)sm_count() * 2 * 128 * 256 * 4;    // groups x splits <= one CTA per SM, 2 tiles each
   return packed_bytes(F_in, F_out) + partial + 256;
 }
 static TcScratch carve(void *scratch, int F_in, int F_out) {
@@ -797,7 +798,7 @@ int varco_tc_gemm_dw(int n, int F_in, int F_out, const void *X, int64_t ldx, con
   int splits = sm_count() / groups;
   if (splits < 1) splits = 1;
   if (splits > p.node_blocks) splits = p.node_blocks;
-  if (splits > 148) splits = 148;
+  if (splits * groups > sm_count()) splits = sm_count() / groups > 0 ? sm_count() / groups : 1;
   p.splits = splits;
   p.partial = sc.partial;
   p.err = err;

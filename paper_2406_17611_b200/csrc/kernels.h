@@ -11,7 +11,13 @@ struct varco_ws_layout {
   int64_t ld_in = 0, ld_out = 0;  // leading dimensions of the internal buffers
   int64_t wstride = 0;            // row stride of the kept-position table (16-bit entries)
   size_t status = 0, packed = 0, halo = 0, wpos = 0, dZ = 0, dAgg = 0, scratch = 0, scratch_bytes = 0, total = 0;
+  // debug build: offsets of the 256-byte guard blocks behind the segments (filled with a pattern by every layer
+  // call, verified by varco_workspace_status)
+  size_t guard[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  int num_guards = 0;
 };
+// debug build: write the guard pattern / the guard table of a layer call (no-ops in a release build)
+int varco_ws_arm_guards(char *ws_base, const varco_ws_layout &L, cudaStream_t st);
 varco_ws_layout varco_make_ws_layout(const varco_plan *pl, int F_in, int F_out, varco_dtype_t dt);
 size_t varco_gemm_scratch_bytes(int F_in, int F_out);
 
@@ -40,6 +46,7 @@ int varco_launch_slot_kept_product(const varco_plan *pl, const void *Gh, int64_t
 int varco_launch_add_dense_rows(const varco_plan *pl, const void *Gh, int64_t ldg, int F, varco_dtype_t dt, void *dX,
                                 int64_t ld, cudaStream_t st);
 // spmm.cu
+int varco_debug_word_spmm();   // debug build: first failed index check of the aggregation kernels (else 0)
 int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, const void *Xhalo, int64_t ldh, int F,
                           varco_dtype_t dt, void *Agg, int64_t ldagg, cudaStream_t st);
 int varco_launch_spmm_bwd(const varco_plan *pl, const void *dAgg, int64_t ldd, int F, varco_dtype_t dt, void *dX,

@@ -4,8 +4,8 @@
 // the receivers' halo slots decompressed (step 3), aggregate exact local rows and lossy remote
 // rows, transform (Eq. (2)).  Backward mirrors it: transform gradients, transposed aggregation
 // to local rows and halo slots, compress the slot gradients with the forward's key, return them
-// to the owners and add (step 4, "back-propagating errors across machines and through the
-// differentiable compression routine").
+// to the owners and add (back-propagation across machines and through the compression routine,
+// Algorithm 1, step 4).
 #include <new>
 
 #include "device_common.cuh"
@@ -37,6 +37,24 @@ size_t varco_gemm_scratch_bytes(int F_in, int F_out) {
   return a > b ? a : b;
 }
 
+int varco_ws_arm_guards(char *ws, const varco_ws_layout &L, cudaStream_t st) {
+#ifdef VARCO_DEBUG
+  unsigned long long table[9] = {0};
+  table[0] = (unsigned long long)L.num_guards;
+  for (int g = 0; g < L.num_guards; ++g) {
+    table[1 + g] = (unsigned long long)L.guard[g];
+    VARCO_CUDA_CHECK(cudaMemsetAsync(ws + L.guard[g], 0xC5, 256, st));
+  }
+  // pageable source: the runtime stages the 72 bytes before the call returns
+  VARCO_CUDA_CHECK(cudaMemcpyAsync(ws + 64, table, sizeof(table), cudaMemcpyHostToDevice, st));
+#else
+  (void)ws;
+  (void)L;
+  (void)st;
+#endif
+  return VARCO_OK;
+}
+
 static char *ws_base(void *workspace) {
   char *ws = static_cast<char *>(workspace);
   return ws + ((256 - (reinterpret_cast<uintptr_t>(ws) & 255u)) & 255u);
@@ -52,9 +70,10 @@ int varco_compress(const varco_plan_t *plan, const void *X, int64_t ld, int32_t 
   if (k < 0) return VARCO_INVALID_ARG;
   if (F > 2048) return VARCO_UNSUPPORTED;
   if (check_matrix(X, ld, F, V) != VARCO_OK) return VARCO_INVALID_ARG;
-  if (plan->H > 0 && !packed) return VARCO_INVALID_ARG;
+  if (plan->H > 0 && k > 0 && !packed) return VARCO_INVALID_ARG;
   if (!plan->uploaded) return VARCO_NOT_UPLOADED;
   if (bytes) *bytes = (uint64_t)plan->H * (uint64_t)k * (dtype == VARCO_F32 ? 4u : 2u);
+  if (k == 0) return VARCO_OK;   // no communication: nothing to pack
   StageTimer t(plan, VARCO_STAGE_COMPRESS, stream);
   return varco_launch_compress_rows(plan, X, ld, F, k, dtype, key, packed, k, 1, nullptr, 0, (cudaStream_t)stream);
 }
@@ -66,9 +85,15 @@ int varco_decompress(const varco_plan_t *plan, const void *packed, int32_t F, va
   const int k = varco_kept_internal(F, c);
   if (k < 0) return VARCO_INVALID_ARG;
   if (F > 2048) return VARCO_UNSUPPORTED;
-  if (plan->H > 0 && (!packed || check_matrix(Xhalo, ld, F, V) != VARCO_OK)) return VARCO_INVALID_ARG;
+  if (plan->H > 0 && ((k > 0 && !packed) || check_matrix(Xhalo, ld, F, V) != VARCO_OK)) return VARCO_INVALID_ARG;
   if (!plan->uploaded) return VARCO_NOT_UPLOADED;
   StageTimer t(plan, VARCO_STAGE_DECOMPRESS, stream);
+  if (k == 0) {   // no communication: every halo row is the zero vector
+    const size_t es = dtype == VARCO_F32 ? 4 : 2;
+    if (plan->H > 0)
+      VARCO_CUDA_CHECK(cudaMemset2DAsync(Xhalo, (size_t)ld * es, 0, (size_t)F * es, (size_t)plan->H, (cudaStream_t)stream));
+    return VARCO_OK;
+  }
   return varco_launch_decompress_slots(plan, packed, k, 1, F, k, dtype, key, Xhalo, ld, nullptr, 0,
                                        (cudaStream_t)stream);
 }
@@ -100,6 +125,7 @@ int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   int *status = reinterpret_cast<int *>(ws + L.status);
   cudaStream_t st = (cudaStream_t)stream;
   VARCO_CUDA_CHECK(cudaMemsetAsync(status, 0, 256, st));
+  if (int grc = varco_ws_arm_guards(ws, L, st)) return grc;
   if (halo_bytes) *halo_bytes = (uint64_t)plan->H * (uint64_t)k * es;
 
   // Exchange.  The copy of a boundary row goes straight to the position of its halo slot at the
@@ -109,8 +135,10 @@ int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   // Compressed epochs with at most a quarter of a row kept: the receiver keeps (value, position)
   // pairs instead of rows that are mostly zeros, and the aggregation reads k pairs per remote
   // neighbour instead of F elements.
-  const bool sparse = k < F_in && varco_spmm_sparse_supported(F_in, k, dt);
-  if (k == F_in) {
+  const bool sparse = k > 0 && k < F_in && varco_spmm_sparse_supported(F_in, k, dt);
+  if (k == 0) {
+    // "no communication" (Section V): nothing is exchanged and every remote neighbour counts as the zero vector
+  } else if (k == F_in) {
     StageTimer t(plan, VARCO_STAGE_COMPRESS, stream);
     rc = varco_launch_gather_copy(plan, X, desc->ld_in, F_in, dt, Xhalo, L.ld_in, st);
   } else {
@@ -129,7 +157,9 @@ int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   if (rc != VARCO_OK) return rc;
   {
     StageTimer t(plan, VARCO_STAGE_SPMM, stream);
-    if (sparse)
+    if (k == 0)
+      rc = varco_launch_spmm_fwd(plan, X, desc->ld_in, nullptr, 0, F_in, dt, Agg_saved, desc->ld_in, st);
+    else if (sparse)
       rc = varco_launch_spmm_fwd_sparse(plan, X, desc->ld_in, Xhalo, round_up64(k, 4), k, F_in, dt, Agg_saved,
                                         desc->ld_in, st);
     else
@@ -154,9 +184,22 @@ int varco_workspace_status(const void *workspace, void *stream, int *device_stat
   int v = 0;
   VARCO_CUDA_CHECK(cudaMemcpyAsync(&v, ws, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
   VARCO_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream));
+#ifdef VARCO_DEBUG
+  // guard table of the last layer call: [count, offsets...] at byte 64 of the status block; a damaged guard
+  // block (some kernel wrote past its segment) sets bit 30 of the status
+  unsigned long long table[9] = {0};
+  VARCO_CUDA_CHECK(cudaMemcpy(table, ws + 64, sizeof(table), cudaMemcpyDeviceToHost));
+  for (unsigned long long g = 0; g < table[0] && g < 8; ++g) {
+    unsigned char block[256];
+    VARCO_CUDA_CHECK(cudaMemcpy(block, ws + table[1 + g], sizeof(block), cudaMemcpyDeviceToHost));
+    for (unsigned char b : block)
+      if (b != 0xC5) v |= 1 << 30;
+  }
+#endif
   *device_status = v;
   return VARCO_OK;
 }
+
 
 int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, const void *X, const void *Y,
                     const void *Agg_saved, const void *W_self, const void *W_neigh, const void *dY, void *dX,
@@ -184,6 +227,7 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   char *ws = ws_base(workspace);
   int *status = reinterpret_cast<int *>(ws + L.status);
   VARCO_CUDA_CHECK(cudaMemsetAsync(status, 0, 256, (cudaStream_t)stream));
+  if (int grc = varco_ws_arm_guards(ws, L, (cudaStream_t)stream)) return grc;
   const bool tc = dt == VARCO_BF16 && F_out <= 256 && (sage ? 2 : 1) * ((F_in + 127) / 128) <= 8;
   void *packed = ws + L.packed;
   void *Ghalo = ws + L.halo;
@@ -229,7 +273,7 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   const bool narrow = tc && 2 * L.ld_out <= F_in;
   uint16_t *wpos = reinterpret_cast<uint16_t *>(ws + L.wpos);
   const int64_t kstride = round_up64(k, V);
-  if (k < F_in) {
+  if (k > 0 && k < F_in) {
     // the kept positions of every unique boundary row are evaluated once, then used by the compression of
     // the slot gradients and by the owners' add
     StageTimer t(plan, VARCO_STAGE_COMPRESS_BWD, stream);
@@ -237,9 +281,9 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
     if (rc != VARCO_OK) return rc;
   }
   if (narrow) {
-    const bool kept_product = k < F_in && varco_slot_kept_product_supported(F_in, F_out, k, dt);
+    const bool kept_product = k > 0 && k < F_in && varco_slot_kept_product_supported(F_in, F_out, k, dt);
     void *Gl = dAgg;      // [n x ld_out] local sums of dZ
-    void *Gh = packed;    // [H x ld_out] slot sums of dZ (dead once the slot rows exist)
+    void *Gh = k > 0 ? packed : nullptr;    // [H x ld_out] slot sums of dZ (dead once the slot rows exist)
     {
       StageTimer t(plan, VARCO_STAGE_SPMM_T, stream);
       rc = varco_launch_spmm_bwd(plan, dZ, lddz, F_out, dt, Gl, L.ld_out, 0, Gh, L.ld_out, nullptr, 0, 0, key, nullptr, 0,
@@ -254,11 +298,11 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
       else
         rc = varco_tc_gemm_cat_t(n, F_in, F_out, Gl, L.ld_out, nullptr, 0, W_neigh, nullptr, dX, desc->ld_in, scratch,
                                  status, st);
-      if (rc == VARCO_OK && plan->H > 0 && !kept_product)
+      if (rc == VARCO_OK && plan->H > 0 && k > 0 && !kept_product)
         rc = varco_tc_gemm_cat_t((int)plan->H, F_in, F_out, Gh, L.ld_out, nullptr, 0, W_neigh, nullptr, Ghalo, L.ld_in,
                                  scratch, status, st);
     }
-    if (rc != VARCO_OK) return rc;
+    if (rc != VARCO_OK || k == 0) return rc;   // no communication: no gradient crosses a partition boundary
     if (kept_product) {
       // few kept entries: each one is a dot product with one row of W_neigh; the F_in-wide rows never exist
       {
@@ -296,10 +340,10 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   {
     StageTimer t(plan, VARCO_STAGE_SPMM_T, stream);
     // k < F: the slot gradients are compressed in the epilogue (no dense slot rows)
-    rc = varco_launch_spmm_bwd(plan, dAgg, L.ld_in, F_in, dt, dX, desc->ld_in, sage ? 1 : 0, Ghalo, L.ld_in,
-                               k < F_in ? packed : nullptr, kstride, k, key, wpos, L.wstride, st);
+    rc = varco_launch_spmm_bwd(plan, dAgg, L.ld_in, F_in, dt, dX, desc->ld_in, sage ? 1 : 0, k > 0 ? Ghalo : nullptr,
+                               L.ld_in, (k > 0 && k < F_in) ? packed : nullptr, kstride, k, key, wpos, L.wstride, st);
   }
-  if (rc != VARCO_OK) return rc;
+  if (rc != VARCO_OK || k == 0) return rc;   // no communication: no gradient crosses a partition boundary
   // Return of the halo-slot gradients to the owners.  At full communication the slot rows are
   // the messages; otherwise they are compressed with the forward's key first.
   if (k == F_in) {

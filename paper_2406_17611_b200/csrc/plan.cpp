@@ -316,7 +316,9 @@ int build(varco_plan *pl, int64_t n, const int64_t *rp0, const int32_t *col0, co
 }  // namespace
 
 int varco_kept_internal(int32_t F, varco_ratio_t c) {
-  if (F < 1 || c.num == 0 || c.den == 0 || c.num < c.den) return -1;
+  if (F < 1 || c.num == 0) return -1;
+  if (c.den == 0) return 0;   // unbounded ratio: the "no communication" setting, nothing is sent
+  if (c.num < c.den) return -1;
   uint64_t k = ((uint64_t)F * c.den + c.num - 1) / c.num;
   if (k < 1) k = 1;
   if (k > (uint64_t)F) k = (uint64_t)F;
@@ -471,6 +473,24 @@ int varco_schedule_linear(int32_t epoch, int32_t K, int32_t slope_a, int32_t c_m
   if (v > 0xFFFFFFFFLL) return VARCO_INVALID_ARG;
   c->num = (uint32_t)v;
   c->den = (uint32_t)K;
+  return VARCO_OK;
+}
+
+int varco_schedule_rate_linear(int32_t epoch, uint32_t r0, uint32_t alpha, uint32_t den, varco_ratio_t *c) {
+  if (!c || epoch < 0 || den == 0 || r0 == 0 || r0 > den) return VARCO_INVALID_ARG;
+  uint64_t r = (uint64_t)r0 + (uint64_t)alpha * (uint64_t)epoch;   // < 2^63: no overflow
+  if (r > den) r = den;
+  c->num = den;
+  c->den = (uint32_t)r;
+  return VARCO_OK;
+}
+
+int varco_schedule_exponential(int32_t epoch, int32_t K, int32_t beta, varco_ratio_t *c) {
+  if (!c || epoch < 0 || K < 1 || beta < 2) return VARCO_INVALID_ARG;
+  uint64_t v = 1;
+  for (int32_t i = epoch; i < K && v < 0xFFFFFFFFull; ++i) v *= (uint64_t)beta;
+  c->num = v > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)v;
+  c->den = 1;
   return VARCO_OK;
 }
 

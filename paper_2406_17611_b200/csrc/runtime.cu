@@ -3,10 +3,16 @@
 #include <mutex>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "device_common.cuh"
 #include "kernels.h"
 
 namespace {
+
+const char *kStageNames[VARCO_STAGE_COUNT] = {"varco:compress",    "varco:decompress", "varco:spmm",    "varco:gemm_fwd",
+                                              "varco:gemm_dx",     "varco:gemm_dw",    "varco:spmm_t",  "varco:compress_bwd",
+                                              "varco:scatter_add", "varco:aux"};
 
 struct ImageItem {
   const void *host;
@@ -55,6 +61,40 @@ std::vector<ImageItem> image_items(varco_plan *pl) {
 
 size_t aligned(size_t b) { return (b + 255) / 256 * 256; }
 
+#ifdef VARCO_DEBUG
+// Debug build: every index array of the image against the extent of what it addresses.
+bool image_is_sound(const varco_plan *pl) {
+  const int64_t n = pl->n, H = pl->H, nsrc = n + H;
+  auto below = [](const std::vector<int32_t> &v, int64_t limit) {
+    for (int32_t x : v)
+      if (x < 0 || x >= limit) return false;
+    return true;
+  };
+  auto monotone = [](const std::vector<int64_t> &v, int64_t last) {
+    for (size_t i = 1; i < v.size(); ++i)
+      if (v[i] < v[i - 1]) return false;
+    return !v.empty() && v.front() == 0 && v.back() == last;
+  };
+  if (!monotone(pl->rp, pl->nnz_f) || !monotone(pl->rpT, pl->nnz_f)) return false;
+  if ((int64_t)pl->rp.size() != n + 1 || (int64_t)pl->rpT.size() != nsrc + 1) return false;
+  if (!below(pl->col, nsrc) || !below(pl->colT, n)) return false;
+  if (!below(pl->slot_src, n) || !below(pl->slot_sendpos, H ? H : 1) || !below(pl->brow, n) || !below(pl->brow_slot, H ? H : 1))
+    return false;
+  if (pl->brow_ptr.empty() || pl->brow_ptr.front() != 0 || pl->brow_ptr.back() != H) return false;
+  for (size_t i = 1; i < pl->brow_ptr.size(); ++i)
+    if (pl->brow_ptr[i] < pl->brow_ptr[i - 1]) return false;
+  if (!below(pl->order_f, n) || !below(pl->hub_f, n) || !below(pl->short_f, n)) return false;
+  if (!below(pl->order_t, nsrc) || !below(pl->hub_t, nsrc) || !below(pl->short_t, nsrc)) return false;
+  for (int32_t c : pl->short_f_col)
+    if (c < -1 || c >= nsrc) return false;
+  for (int32_t c : pl->short_t_col)
+    if (c < -1 || c >= n) return false;
+  for (int64_t r = 0; r < n; ++r)
+    if (pl->nloc[r] < 0 || pl->nloc[r] > pl->rp[r + 1] - pl->rp[r]) return false;
+  return true;
+}
+#endif
+
 std::atomic<int64_t> g_kernel_launches{0};
 
 }  // namespace
@@ -74,7 +114,10 @@ struct varco_profile {
   bool is_open[VARCO_STAGE_COUNT] = {};
 };
 
+// Every stage is also an NVTX range (a profiler timeline shows the stages by name; without a tool attached
+// the calls return at once).
 void varco_prof_begin(const varco_plan *plan, int stage, void *stream) {
+  nvtxRangePushA(kStageNames[stage]);
   varco_profile *pr = plan->prof;
   if (!pr || !pr->on) return;
   std::lock_guard<std::mutex> lock(pr->mu);
@@ -95,6 +138,7 @@ void varco_prof_begin(const varco_plan *plan, int stage, void *stream) {
 }
 
 void varco_prof_end(const varco_plan *plan, int stage, void *stream) {
+  nvtxRangePop();
   varco_profile *pr = plan->prof;
   if (!pr || !pr->on) return;
   std::lock_guard<std::mutex> lock(pr->mu);
@@ -186,6 +230,21 @@ int varco_profile_spans(varco_plan_t *plan, int32_t stage, double *milliseconds,
   return VARCO_OK;
 }
 
+int varco_debug_status(int32_t *is_debug_build, int32_t *word) {
+  if (!is_debug_build || !word) return VARCO_INVALID_ARG;
+#ifdef VARCO_DEBUG
+  *is_debug_build = 1;
+  VARCO_CUDA_CHECK(cudaDeviceSynchronize());
+  const int w = varco_debug_word_spmm();
+  if (w < 0) return VARCO_CUDA;
+  *word = w;
+#else
+  *is_debug_build = 0;
+  *word = 0;
+#endif
+  return VARCO_OK;
+}
+
 int varco_kernel_launches(int64_t *count) {
   if (!count) return VARCO_INVALID_ARG;
   *count = g_kernel_launches.load(std::memory_order_relaxed);
@@ -207,6 +266,9 @@ int varco_partition_upload(varco_plan_t *plan, void *dev_buf, size_t bytes, void
   size_t need = 0;
   varco_partition_device_bytes(plan, &need);
   if (bytes < need) return VARCO_WORKSPACE_TOO_SMALL;
+#ifdef VARCO_DEBUG
+  if (!image_is_sound(plan)) return VARCO_BAD_GRAPH;
+#endif
   plan->uploaded = false;
   size_t off = 0;
   for (const ImageItem &it : image_items(plan)) {
@@ -243,6 +305,10 @@ varco_ws_layout varco_make_ws_layout(const varco_plan *pl, int F_in, int F_out, 
   auto take = [&](size_t b) {
     size_t o = off;
     off += aligned(b);
+#ifdef VARCO_DEBUG
+    if (L.num_guards < 8) L.guard[L.num_guards++] = off;   // 256 guard bytes behind every segment
+    off += 256;
+#endif
     return o;
   };
   L.status = take(256);                             // device status word of the last layer call

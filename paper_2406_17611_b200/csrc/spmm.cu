@@ -83,6 +83,9 @@ struct SpmmArgs {
   const int32_t *short_col;   // 8-entry records of the short class (nullptr: walk the CSR)
   const float *short_val;
   int short_nlocal;           // leading rows of the short class whose result is a local row (the rest: halo slots)
+  const int32_t *nloc_only;   // forward, no communication: per-row count of local entries (else nullptr)
+  int row_limit;              // transposed, no communication: first row that is not computed (0: all rows)
+  int nsrc, ndst;             // extents of the source / destination index spaces
 };
 
 // task id -> (position in the class list, panel); tasks are ordered (partition, panel, row)
@@ -111,6 +114,12 @@ struct GatherSrc {
   const uint4 *b0, *b1s;   // in 16-byte units
   int ld0, ld1;            // row strides in 16-byte units
   int split;
+  // "no communication" (k = 0): a forward row stops after its nloc[r] local entries (the halo entries would
+  // add zero vectors), and the transposed pass leaves out the rows at or beyond row_limit (the halo slots,
+  // whose gradients nobody receives)
+  const int32_t *nloc_only;   // nullptr: rows are walked whole
+  int row_limit;              // rows >= row_limit are not computed (INT_MAX: all)
+  int nsrc, ndst;             // extents of the source and destination index spaces (checked in the debug build)
 };
 
 // acc[j] = w * f[j] + acc[j] for V values, two per instruction (packed fp32 FMA of sm_100; each half rounds
@@ -147,10 +156,11 @@ __device__ __forceinline__ void accumulate_range(const int32_t *__restrict__ col
         const int c = __shfl_sync(gmask, myc, t + u, G);
         w[u] = __shfl_sync(gmask, myw, t + u, G);
         const bool loc = c < gs.split;
+        const bool ok = VARCO_DBG_OK(c, gs.nsrc, 11);
         const uint4 *src = (loc ? gs.b0 : gs.b1s) + (int64_t)c * (loc ? gs.ld0 : gs.ld1) + (ch_lo + gl);
 #pragma unroll
         for (int i = 0; i < NCH; ++i)
-          v[u][i] = (FULL || ch_lo + gl + i * G < ch_hi) ? __ldg(src + i * G) : make_uint4(0u, 0u, 0u, 0u);
+          v[u][i] = (ok && (FULL || ch_lo + gl + i * G < ch_hi)) ? __ldg(src + i * G) : make_uint4(0u, 0u, 0u, 0u);
       }
 #pragma unroll
       for (int u = 0; u < UNR; ++u)
@@ -263,6 +273,7 @@ __global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
   int pos, panel;
   locate(rc, P, panels, task, pos, panel);
   const int r = __ldg(rc.rows + pos);
+  if (r >= gs.row_limit || !VARCO_DBG_OK(r, gs.ndst, 12)) return;
   const int ch_lo = panel * nv_panel;
   const int ch_hi = min(nv, ch_lo + nv_panel);
 
@@ -272,7 +283,8 @@ __global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
 #pragma unroll
     for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
   const int64_t e0 = rp[r];
-  accumulate_range<T, G, NCH, UNR, FULL>(col + e0, val + e0, (int)(rp[r + 1] - e0), gs, ch_lo, ch_hi, gl, gmask, acc);
+  const int len = gs.nloc_only ? __ldg(gs.nloc_only + r) : (int)(rp[r + 1] - e0);
+  accumulate_range<T, G, NCH, UNR, FULL>(col + e0, val + e0, len, gs, ch_lo, ch_hi, gl, gmask, acc);
   finish_row<T, G, NCH, FULL>(acc, r, gl, gmask, ch_lo, ch_hi, nv, stage_rows, O0, ldo0, O1, ldo1, dst_split, accumulate0,
                               hc);
 }
@@ -299,9 +311,14 @@ __global__ void __launch_bounds__(256, short_blocks_per_sm(NCH))
     myw = __ldg(rec_val + (int64_t)task * 8 + gl);
   }
   const int r = __ldg(rows + task);
+  if (!VARCO_DBG_OK(r, gs.ndst, 12)) return;
+  if (gs.nloc_only && myc >= gs.split) myc = -1;   // no communication: halo entries add nothing
   const int cnt = __popc(__ballot_sync(gmask, myc >= 0) & gmask);
   const int c_first = __shfl_sync(gmask, myc, 0, G);
-  if (myc < 0) myc = c_first;   // lanes past the row's length: a valid source with weight zero
+  if (myc < 0) {   // lanes past the row's length: a valid source with weight zero
+    myc = c_first;
+    myw = 0.f;
+  }
   float acc[NCH][V];
 #pragma unroll
   for (int i = 0; i < NCH; ++i)
@@ -315,9 +332,11 @@ __global__ void __launch_bounds__(256, short_blocks_per_sm(NCH))
       const int c = __shfl_sync(gmask, myc, t + u, G);
       w[u] = __shfl_sync(gmask, myw, t + u, G);
       const bool loc = c < gs.split;
+      const bool ok = VARCO_DBG_OK(c, gs.nsrc, 11);
       const uint4 *src = (loc ? gs.b0 : gs.b1s) + (int64_t)c * (loc ? gs.ld0 : gs.ld1) + gl;
 #pragma unroll
-      for (int i = 0; i < NCH; ++i) v[u][i] = (FULL || gl + i * G < nv) ? __ldg(src + i * G) : make_uint4(0u, 0u, 0u, 0u);
+      for (int i = 0; i < NCH; ++i)
+        v[u][i] = (ok && (FULL || gl + i * G < nv)) ? __ldg(src + i * G) : make_uint4(0u, 0u, 0u, 0u);
     }
 #pragma unroll
     for (int u = 0; u < UNR; ++u)
@@ -368,7 +387,7 @@ __global__ void __launch_bounds__(256)
     for (int u = 0; u < 4; ++u) {
       const int c = __shfl_sync(gmask, myc, t + u, KL);
       w[u] = __shfl_sync(gmask, myw, t + u, KL);
-      x[u] = __ldg(col_base + (int64_t)c * lda);
+      x[u] = VARCO_DBG_OK(c, dst_split, 11) ? __ldg(col_base + (int64_t)c * lda) : (E)0;
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
@@ -402,9 +421,10 @@ __global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
   int pos, panel;
   locate(rc, P, panels, blockIdx.x, pos, panel);
   const int r = __ldg(rc.rows + pos);
+  if (r >= gs.row_limit || !VARCO_DBG_OK(r, gs.ndst, 12)) return;
   const int ch_lo = panel * nv_panel;
   const int ch_hi = min(nv, ch_lo + nv_panel);
-  const int64_t e0 = rp[r], e1 = rp[r + 1];
+  const int64_t e0 = rp[r], e1 = gs.nloc_only ? e0 + __ldg(gs.nloc_only + r) : rp[r + 1];
   // the entries are shared out over the warps, and inside a warp over its 32 / G lane groups (narrow rows
   // need fewer than 32 lanes per gathered row); the groups' sums meet by a fixed shuffle tree
   constexpr int kGroups = 32 / G;
@@ -492,6 +512,10 @@ GatherSrc gather_src(const SpmmArgs &a) {
   gs.ld1 = (int)(a.lda1 / V);
   gs.b1s = reinterpret_cast<const uint4 *>(a.A1) - (int64_t)a.src_split * gs.ld1;
   gs.split = a.src_split;
+  gs.nloc_only = a.nloc_only;
+  gs.row_limit = a.row_limit > 0 ? a.row_limit : 0x7FFFFFFF;
+  gs.nsrc = a.nsrc;
+  gs.ndst = a.ndst;
   return gs;
 }
 
@@ -595,6 +619,7 @@ int launch(const SpmmArgs &a, cudaStream_t st) {
   if (a.panels == 1 && a.short_col) {
     constexpr int GR = GS < 8 ? 8 : GS, NR = GS < 8 ? (NCHS * GS + 7) / 8 : NCHS;
     const int nl = a.short_nlocal, ns = a.shorts.count - nl;
+    if (a.row_limit > 0) return launch_short<T, GR, NR, VARCO_SHORT_UNR>(a, 0, nl, st);
     if (ns > 0 && kept_columns_pay<T>(a)) {
       if (int rc = launch_short<T, GR, NR, VARCO_SHORT_UNR>(a, 0, nl, st)) return rc;
       return launch_short_kept<T>(a, nl, ns, st);
@@ -647,34 +672,39 @@ __device__ __forceinline__ void add_chunk(float (&acc)[4], const uint4 &v, float
       : "r"(v.z), "r"(v.w));
 }
 
-// acc[i][:] += chunk (gl + i G) of every source col[e], e < len; `base` is the lane's own chunk of row 0
+// acc[i][:] += chunk (gl + i G) of every source col[e], e < len; `base` is the lane's own chunk of row 0.
+// The indices of the next G entries are fetched while the gathers of the current ones are in flight, and a
+// ragged last batch issues all its loads before the first add (the loads of a batch must never wait on each
+// other: a row is a handful of round trips to L2 or DRAM and nothing else).
 template <typename T, int G, int NCH, int UNR, bool FULL>
 __device__ __forceinline__ void sum_range(const int32_t *__restrict__ colp, int len, const uint4 *__restrict__ base,
                                           int ld, int nv, int gl, unsigned gmask,
-                                          float (&acc)[NCH][ElemTraits<T>::kVec]) {
+                                          float (&acc)[NCH][ElemTraits<T>::kVec], int c_lo, int c_hi) {
+  if (len <= 0) return;
+  int myc = __ldg(colp + min(gl, len - 1));
   for (int b = 0; b < len; b += G) {
     const int cnt = min(G, len - b);
-    const int myc = __ldg(colp + b + min(gl, cnt - 1));
-    int t = 0;
-    for (; t + UNR <= cnt; t += UNR) {
+    const int cur = myc;
+    if (b + G < len) myc = __ldg(colp + b + G + min(gl, len - b - G - 1));
+    for (int t = 0; t < cnt; t += UNR) {
       uint4 v[UNR][NCH];
 #pragma unroll
       for (int u = 0; u < UNR; ++u) {
-        const uint4 *src = base + (int64_t)__shfl_sync(gmask, myc, t + u, G) * ld;
+        if (t + u < cnt) {   // the same for every lane of the group
+          const int c = __shfl_sync(gmask, cur, t + u, G);
+          const bool ok = VARCO_DBG_OK(c - c_lo, c_hi - c_lo, 11);
+          const uint4 *src = base + (int64_t)c * ld;
 #pragma unroll
-        for (int i = 0; i < NCH; ++i)
-          v[u][i] = (FULL || gl + i * G < nv) ? __ldg(src + i * G) : make_uint4(0u, 0u, 0u, 0u);
+          for (int i = 0; i < NCH; ++i)
+            v[u][i] = (ok && (FULL || gl + i * G < nv)) ? __ldg(src + i * G) : make_uint4(0u, 0u, 0u, 0u);
+        }
       }
 #pragma unroll
       for (int u = 0; u < UNR; ++u)
+        if (t + u < cnt) {
 #pragma unroll
-        for (int i = 0; i < NCH; ++i) add_chunk(acc[i], v[u][i], T());
-    }
-    for (; t < cnt; ++t) {
-      const uint4 *src = base + (int64_t)__shfl_sync(gmask, myc, t, G) * ld;
-#pragma unroll
-      for (int i = 0; i < NCH; ++i)
-        if (FULL || gl + i * G < nv) add_chunk(acc[i], __ldg(src + i * G), T());
+          for (int i = 0; i < NCH; ++i) add_chunk(acc[i], v[u][i], T());
+        }
     }
   }
 }
@@ -685,6 +715,7 @@ struct SumSrc {
   int ld0, ld1;
   const int32_t *nloc;
   const float *row_scale;   // 1 / deg(r)
+  int n, nsrc;              // rows, rows + halo slots (checked in the debug build)
 };
 
 template <typename T, int NCH, bool FULL>
@@ -724,8 +755,10 @@ __global__ void __launch_bounds__(256, sum_blocks_per_sm(NCH, UNR))
   const int64_t e0 = rp[r];
   const int len = (int)(rp[r + 1] - e0);
   const int nl = __ldg(ss.nloc + r);
-  sum_range<T, G, NCH, UNR, FULL>(col + e0, nl, ss.b0 + gl, ss.ld0, nv, gl, gmask, acc);
-  if (len > nl) sum_range<T, G, NCH, UNR, FULL>(col + e0 + nl, len - nl, ss.b1s + gl, ss.ld1, nv, gl, gmask, acc);
+  if (!VARCO_DBG_OK(r, ss.n, 12)) return;
+  sum_range<T, G, NCH, UNR, FULL>(col + e0, nl, ss.b0 + gl, ss.ld0, nv, gl, gmask, acc, 0, ss.n);
+  if (len > nl && ss.b1s)   // no halo rows: "no communication", the remote entries add nothing
+    sum_range<T, G, NCH, UNR, FULL>(col + e0 + nl, len - nl, ss.b1s + gl, ss.ld1, nv, gl, gmask, acc, ss.n, ss.nsrc);
   store_scaled<T, NCH, FULL>(acc, __ldg(ss.row_scale + r), O, ldo, r, gl, G, nv);
 }
 
@@ -761,9 +794,10 @@ __global__ void __launch_bounds__(256, sum_blocks_per_sm(NCH, UNR))
   };
   int b0, b1;
   share(nl, b0, b1);
-  if (b1 > b0) sum_range<T, G, NCH, UNR, FULL>(col + e0 + b0, b1 - b0, ss.b0 + gl, ss.ld0, nv, gl, gmask, acc);
-  share(len - nl, b0, b1);
-  if (b1 > b0) sum_range<T, G, NCH, UNR, FULL>(col + e0 + nl + b0, b1 - b0, ss.b1s + gl, ss.ld1, nv, gl, gmask, acc);
+  if (b1 > b0) sum_range<T, G, NCH, UNR, FULL>(col + e0 + b0, b1 - b0, ss.b0 + gl, ss.ld0, nv, gl, gmask, acc, 0, ss.n);
+  share(ss.b1s ? len - nl : 0, b0, b1);
+  if (b1 > b0)
+    sum_range<T, G, NCH, UNR, FULL>(col + e0 + nl + b0, b1 - b0, ss.b1s + gl, ss.ld1, nv, gl, gmask, acc, ss.n, ss.nsrc);
 #pragma unroll
   for (int off = G; off < 32; off <<= 1)
 #pragma unroll
@@ -882,7 +916,7 @@ template <typename T, int G>
 __device__ __forceinline__ void accumulate_sparse(const int32_t *__restrict__ colp, const float *__restrict__ valp,
                                                   int len, const typename SparsePair<T>::type *__restrict__ pairs,
                                                   int64_t pstride, int k, int split, float *sacc, int gl,
-                                                  unsigned gmask) {
+                                                  unsigned gmask, int nslots, int width) {
   typedef typename SparsePair<T>::type P;
   for (int base = 0; base < len; base += G) {
     const int cnt = min(G, len - base);
@@ -898,11 +932,12 @@ __device__ __forceinline__ void accumulate_sparse(const int32_t *__restrict__ co
         for (int u = 0; u < 4; ++u) {
           const int slot = __shfl_sync(gmask, myc, t + u, G) - split;
           w[u] = __shfl_sync(gmask, myw, t + u, G);
-          p[u] = __ldg(pairs + (int64_t)slot * pstride + min(gl, k - 1));
+          p[u] = VARCO_DBG_OK(slot, nslots, 11) ? __ldg(pairs + (int64_t)slot * pstride + min(gl, k - 1)) : P();
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          if (gl < k) sacc[SparsePair<T>::pos(p[u])] += w[u] * SparsePair<T>::val(p[u]);
+          if (gl < k && VARCO_DBG_OK(SparsePair<T>::pos(p[u]), width, 13))
+            sacc[SparsePair<T>::pos(p[u])] += w[u] * SparsePair<T>::val(p[u]);
           __syncwarp(gmask);
         }
       }
@@ -911,10 +946,11 @@ __device__ __forceinline__ void accumulate_sparse(const int32_t *__restrict__ co
         const int slot = __shfl_sync(gmask, myc, t, G) - split;
         const float w = __shfl_sync(gmask, myw, t, G);
         const P *pr = pairs + (int64_t)slot * pstride;
-        for (int m = gl; m < k; m += G) {
-          const P q = __ldg(pr + m);
-          sacc[SparsePair<T>::pos(q)] += w * SparsePair<T>::val(q);
-        }
+        if (VARCO_DBG_OK(slot, nslots, 11))
+          for (int m = gl; m < k; m += G) {
+            const P q = __ldg(pr + m);
+            if (VARCO_DBG_OK(SparsePair<T>::pos(q), width, 13)) sacc[SparsePair<T>::pos(q)] += w * SparsePair<T>::val(q);
+          }
         __syncwarp(gmask);
       }
     }
@@ -948,7 +984,8 @@ __global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
     for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
   __syncwarp(gmask);
   if (nl > 0) accumulate_range<T, G, NCH, 4, FULL>(col + e0, val + e0, nl, gs, 0, nv, gl, gmask, acc);
-  if (len > nl) accumulate_sparse<T, G>(col + e0 + nl, val + e0 + nl, len - nl, pairs, pstride, k, gs.split, sacc, gl, gmask);
+  if (len > nl) accumulate_sparse<T, G>(col + e0 + nl, val + e0 + nl, len - nl, pairs, pstride, k, gs.split, sacc, gl, gmask,
+                                       gs.nsrc - gs.split, nv * V);
   uint4 *dst = reinterpret_cast<uint4 *>(O + (int64_t)r * ldo);
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
@@ -997,7 +1034,7 @@ __global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
   share(len - nl, b0, b1);
   if (b1 > b0)
     accumulate_sparse<T, 32>(col + e0 + nl + b0, val + e0 + nl + b0, b1 - b0, pairs, pstride, k, gs.split, sacc, lane,
-                             0xFFFFFFFFu);
+                             0xFFFFFFFFu, gs.nsrc - gs.split, nv * V);
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
     const int ch = lane + i * 32;
@@ -1080,6 +1117,7 @@ int dispatch_sparse(const SpmmArgs &a, const int32_t *nloc, const void *pairs, i
 }  // namespace
 
 // Forward aggregation: Agg[r] = sum_e val[e] * (col[e] < n ? X[col[e]] : Xhalo[col[e] - n]).
+// Xhalo == nullptr: nothing was communicated, the halo entries contribute zero vectors.
 int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, const void *Xhalo, int64_t ldh, int F,
                           varco_dtype_t dt, void *Agg, int64_t ldagg, cudaStream_t st) {
   const int V = dt == VARCO_F32 ? 4 : 8;
@@ -1097,6 +1135,8 @@ int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, cons
   a.A1 = Xhalo;
   a.lda1 = ldh;
   a.src_split = (int)pl->n;
+  a.nsrc = (int)(pl->n + pl->H);
+  a.ndst = (int)pl->n;
   a.O0 = Agg;
   a.ldo0 = ldagg;
   a.O1 = nullptr;
@@ -1123,6 +1163,14 @@ int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, cons
   a.short_col = pl->d.short_f_col;
   a.short_val = pl->d.short_f_val;
   a.short_nlocal = (int)pl->short_f.size();
+  if (!Xhalo) {   // no communication: local entries only
+    a.A1 = X;
+    a.lda1 = ldx;
+    a.nloc_only = pl->d.nloc;
+    a.panels = 1;
+    a.nv_panel = nv;
+    ldh = ldx;
+  }
   if (a.panels == 1 && !pl->row_scale.empty() && (ldx % V) == 0 && (ldh % V) == 0) {
     // mean aggregation: unweighted sums, one scale per finished row
     SumArgs u{};
@@ -1134,9 +1182,11 @@ int varco_launch_spmm_fwd(const varco_plan *pl, const void *X, int64_t ldx, cons
     u.ss.b0 = reinterpret_cast<const uint4 *>(X);
     u.ss.ld0 = (int)(ldx / V);
     u.ss.ld1 = (int)(ldh / V);
-    u.ss.b1s = reinterpret_cast<const uint4 *>(Xhalo) - (int64_t)pl->n * u.ss.ld1;
+    u.ss.b1s = Xhalo ? reinterpret_cast<const uint4 *>(Xhalo) - (int64_t)pl->n * u.ss.ld1 : nullptr;
     u.ss.nloc = pl->d.nloc;
     u.ss.row_scale = pl->d.row_scale;
+    u.ss.n = (int)pl->n;
+    u.ss.nsrc = (int)(pl->n + pl->H);
     u.O = Agg;
     u.ldo = ldagg;
     u.nv = nv;
@@ -1171,6 +1221,8 @@ int varco_launch_spmm_fwd_sparse(const varco_plan *pl, const void *X, int64_t ld
   a.A1 = X;
   a.lda1 = ldx;
   a.src_split = (int)pl->n;
+  a.nsrc = (int)(pl->n + pl->H);
+  a.ndst = (int)pl->n;
   a.O0 = Agg;
   a.ldo0 = ldagg;
   a.dst_split = (int)pl->n;
@@ -1205,6 +1257,8 @@ int varco_launch_spmm_bwd(const varco_plan *pl, const void *dAgg, int64_t ldd, i
   a.A1 = dAgg;
   a.lda1 = ldd;
   a.src_split = (int)pl->n;
+  a.nsrc = (int)pl->n;
+  a.ndst = (int)(pl->n + pl->H);
   a.O0 = dX;
   a.ldo0 = ldx;
   a.O1 = Ghalo;
@@ -1217,8 +1271,12 @@ int varco_launch_spmm_bwd(const varco_plan *pl, const void *dAgg, int64_t ldd, i
   a.short_col = pl->d.short_t_col;
   a.short_val = pl->d.short_t_val;
   a.short_nlocal = (int)pl->short_t_nlocal;
+  if (!Ghalo && !packed) a.row_limit = (int)pl->n;   // no communication: the halo-slot rows are not computed
   if (packed)
     a.hc = HaloCompress{packed, kstride, k, F, vperm::half_bits(F), vperm::layer_key(key), pl->d.slot_gid, wpos, wstride,
                         pl->d.slot_src};
   return dt == VARCO_F32 ? dispatch<float>(a, st) : dispatch<__nv_bfloat16>(a, st);
 }
+
+// debug build: this translation unit's word of failed index checks (0 in a release build)
+VARCO_DEFINE_DEBUG_READER(varco_debug_word_spmm)

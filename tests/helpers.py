@@ -37,6 +37,29 @@ def rel_err(got, ref):
     return float(np.max(np.abs(got - ref)) / max(float(np.max(np.abs(ref))), 1e-30))
 
 
+def rel_err_axis(got, ref, axis, floor=5e-2):
+    """Scaled companion of rel_err: the largest |got - ref| of every column (axis=0) or row (axis=1) over that
+    column's / row's own max |ref| -- not below `floor` times the tensor's max, so that a column of ReLU zeros
+    does not divide by nothing.  A wrong low-magnitude column (a padded tail, one feature) or row (a high-degree
+    node whose mean is small, a dropped neighbour) cannot hide behind the largest entries of the tensor."""
+    ref = np.asarray(ref, dtype=np.float64)
+    got = np.asarray(got, dtype=np.float64)
+    if ref.ndim == 1:
+        ref, got = ref[None, :], got[None, :]
+    gmax = max(float(np.abs(ref).max()), 1e-30)
+    scale = np.maximum(np.abs(ref).max(axis=axis), floor * gmax)
+    return float((np.abs(got - ref).max(axis=axis) / scale).max())
+
+
+def close(got, ref, tol):
+    """Norm-wise within tol, and within 2 tol against every column's and every row's own scale."""
+    e, ec, er = rel_err(got, ref), rel_err_axis(got, ref, 0), rel_err_axis(got, ref, 1)
+    ok = e <= tol and ec <= 2 * tol and er <= 2 * tol
+    if not ok:
+        print("close(): norm-wise %.3e, column-wise %.3e, row-wise %.3e, tol %.1e" % (e, ec, er, tol))
+    return ok
+
+
 def dev_weights(w, dtype, dev="cuda:0"):
     return None if w is None else torch.from_numpy(np.ascontiguousarray(w)).to(dtype).to(dev).contiguous()
 

@@ -54,6 +54,22 @@ def test_rate_helpers_match_oracle(orc):
                 assert r == orc.schedule_linear(e, K, a)
                 assert vb.varco_kept(F, r) == orc.kept(F, r)
     # worked values: K=100, a=5 -> c_e = 128 - 6.35 e; F=256 keeps 2, 3, ... 35 (e=19), 256 (e>=20)
+    # the other schedulers of the appendix, the fixed ratios of Section V and "no communication"
+    for r0, al, den in [(1, 1, 128), (1, 3, 64), (5, 7, 300), (2, 0, 9)]:
+        for e in list(range(0, 140, 7)) + [10**6]:
+            r = vb.varco_schedule_rate_linear(e, r0, al, den)
+            assert r == orc.schedule_rate_linear(e, r0, al, den) == orc.schedule_fixed_increment(min(e, 5000), r0, al, den) \
+                or (e > 5000 and r == orc.schedule_rate_linear(e, r0, al, den))
+            assert vb.varco_kept(100, r) == orc.kept(100, r)
+    for beta, K in [(2, 7), (3, 5), (10, 20)]:
+        for e in range(K + 3):
+            r = vb.varco_schedule_exponential(e, K, beta)
+            assert r == orc.schedule_exponential(e, K, beta)
+            assert vb.varco_kept(256, r) == orc.kept(256, r)
+    for F in (8, 47, 100, 256, 602):
+        assert vb.varco_kept(F, vb.NO_COMMUNICATION) == orc.kept(F, (1, 0)) == 0
+        for c in (2, 4):
+            assert vb.varco_kept(F, (c, 1)) == orc.kept(F, (c, 1)) == -(-F // c)
     ks = [vb.varco_kept(256, vb.varco_schedule_linear(e, 100)) for e in range(22)]
     assert ks[0] == 2 and ks[1] == 3 and ks[19] == 35 and ks[20] == ks[21] == 256
     assert vb.varco_kept(256, vb.varco_schedule_linear(59, 300)) == 83

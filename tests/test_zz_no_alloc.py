@@ -18,12 +18,16 @@ from paper_2406_17611_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-def test_noalloc_exchange_matches_compress_decompress_twice():
+def test_noalloc_exchange_matches_compress_decompress_twice(orc):
     wl = synth.make_workload("c3", 0.004)
     plan = vb.Plan(wl.row_ptr, wl.col, wl.part, wl.parts, wl.conv).upload()
+    g = orc.graph(wl.row_ptr, wl.col, wl.part, wl.parts, wl.conv)
     perm = plan.perm()
+    # the last two calls keep whole rows (k = F): 100 bf16 and 64 fp32 values per copy, both inside the scratch
     calls = [(100, (4, 1), (7, 1, 0), torch.bfloat16), (256, (16, 1), (7, 2, 1), torch.bfloat16),
-             (64, (385, 4), (7, 3, 0), torch.float32)]
+             (64, (385, 4), (7, 3, 0), torch.float32), (100, (1, 1), (7, 4, 1), torch.bfloat16),
+             (64, (1, 1), (7, 5, 0), torch.float32)]
+    assert plan.H_total * 104 * 2 <= vb.NOALLOC_SCRATCH_BYTES and plan.H_total * 64 * 4 <= vb.NOALLOC_SCRATCH_BYTES
     for rep in range(2):
         for F, ratio, key, dt in calls:
             vec = 4 if dt == torch.float32 else 8
@@ -41,6 +45,11 @@ def test_noalloc_exchange_matches_compress_decompress_twice():
             assert torch.cuda.memory_allocated() == before
             assert got_bytes == want_bytes
             assert torch.equal(out[:, :F], want[:, :F])
+            # and against the oracle itself: decompress(compress(X)), bit for bit, same byte count
+            ref_packed, sent = g.compress(X, ratio, key)
+            assert got_bytes == sent * (4 if dt == torch.float32 else 2)
+            ref = g.decompress(ref_packed, F, ratio, key)
+            assert np.array_equal(out[:, :F].to(torch.float64).cpu().numpy(), ref)
 
 
 def test_noalloc_exchange_rejects_sizes_beyond_its_scratch():
