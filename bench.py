@@ -617,6 +617,22 @@ def q_sweep(args, wl0, device, ratio):
                        "nnz": wl0.nnz, "steps": args.steps}}
 
 
+def max_over_ranks(ms, world, device=None):
+    """The slowest rank's time: what a multi-rank number is quoted on (all-reduce MAX; identity on one rank)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(units_per_rank, ms_per_step, world):
+    """Whole-job throughput of `world` replicas that each process `units_per_rank` per step."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
+
+
 # ------------------------------------------------------------------------------------------ ours
 def run_ours(args):
     import torch
@@ -677,13 +693,10 @@ def run_ours(args):
     spans_keep = {st: model.plan.profile_spans(st) for st in ("gemm_fwd", "gemm_dx", "gemm_dw")}
     model.plan.profile_enable(False)
     model.plan.profile_reset()
-    if world > 1:
-        t = torch.tensor([ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, device)
     ms_per_step = ms / args.steps
     edges_per_step = wl.nnz * L
-    value = world * edges_per_step / (ms_per_step * 1e-3)
+    value = aggregate_value(edges_per_step, ms_per_step, world)
 
     # end to end: inputs from pinned host memory, results back to the host, inside the timed region
     e2e = None
@@ -701,12 +714,9 @@ def run_ours(args):
         barrier()
         wall_ms = 1e3 * (time.perf_counter() - t_host)
         ms_e2e = max(e0.elapsed_time(e1), 0.0)
-        if world > 1:
-            t = torch.tensor([ms_e2e], device=device, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e = max_over_ranks(ms_e2e, world, device)
         h2d, d2h = model.e2e_bytes()
-        e2e = {"value": world * edges_per_step / (ms_e2e / n_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": aggregate_value(edges_per_step, ms_e2e / n_e2e, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / n_e2e, "host_wall_ms_per_step": wall_ms / n_e2e}
 
     if rank != 0:

@@ -134,3 +134,40 @@ def test_gather_model_matches_brute_force():
             e, s_, r = plan.gather_model(keep, transposed)
             assert (e, s_, r) == (int(cnt.sum()), len(cnt), want)
     plan.close()
+
+
+def test_halo_bytes_of_the_100_epoch_schedule_follow_the_closed_form(orc):
+    """The rate-sweep configuration (4-layer SAGE 100-256-256-256-47, bf16, schedule K = 100, slope 5): for every
+    epoch the bytes of one epoch, forward and backward, are 2 * sum_l H_total * k_l * s -- the library's plan
+    and rate helpers against the oracle's, all 100 epochs; and the oracle's own byte counter (which counts values
+    as they are sent) agrees with the closed form at the schedule's corner epochs."""
+    wl = synth.make_workload("c5", 0.001)
+    plan = vb.Plan(wl.row_ptr, wl.col, wl.part, wl.parts, wl.conv)
+    g = orc.graph(wl.row_ptr, wl.col, wl.part, wl.parts, wl.conv)
+    assert plan.H_total == g.H_total
+    widths, es = wl.widths, 2
+    total_lib = total_orc = 0
+    for e in range(100):
+        r = vb.varco_schedule_linear(e, 100, 5)
+        assert r == orc.schedule_linear(e, 100, 5)
+        ks = [vb.varco_kept(F, r) for F in widths[:-1]]
+        assert ks == [orc.kept(F, r) for F in widths[:-1]]
+        total_lib += 2 * sum(plan.H_total * k * es for k in ks)
+        total_orc += 2 * sum(g.H_total * orc.kept(F, r) * es for F in widths[:-1])
+        if e >= 20:
+            assert ks == widths[:-1]                       # full communication from epoch K / a on
+    assert total_lib == total_orc
+    full = 2 * sum(plan.H_total * F * es for F in widths[:-1])
+    assert total_lib < 100 * full and total_lib > 80 * full
+    for e in (0, 1, 19, 20):
+        r = orc.schedule_linear(e, 100, 5)
+        sent = 0
+        for l in range(4):
+            X = synth.normal_features(wl.n, widths[l], 3, True)
+            Ws, Wn, b = wl.layer_weights(l)
+            Y, _, hb = g.layer_fwd(X, Ws, Wn, b, l < 3, r, (1, e, l), elem_bytes=es)
+            dY = np.ones((wl.n, widths[l + 1]))
+            hb2 = g.layer_bwd(X, Y, Ws, Wn, dY, l < 3, r, (1, e, l), elem_bytes=es)[4]
+            sent += hb + hb2
+        assert sent == 2 * sum(g.H_total * orc.kept(F, r) * es for F in widths[:-1])
+    plan.close()

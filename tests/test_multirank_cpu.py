@@ -10,19 +10,18 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 WORKER = r"""
 import os, sys, json
-import torch, torch.distributed as dist
+import torch.distributed as dist
 sys.path.insert(0, %r)
+import bench                         # the benchmark's own reduction and aggregation, on the gloo backend
 dist.init_process_group("gloo")
 rank, world = dist.get_rank(), dist.get_world_size()
 # every rank holds its own replica's step time; the reported time is the max over ranks and the
 # reported throughput the sum of the replicas' work over that time
-ms = torch.tensor([10.0 + 5.0 * rank], dtype=torch.float64)
 dist.barrier()
-dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-edges = 1000
-value = world * edges / (ms.item() * 1e-3)
+ms = bench.max_over_ranks(10.0 + 5.0 * rank, world)
+value = bench.aggregate_value(1000, ms, world)
 if rank == 0:
-    print(json.dumps({"ms": ms.item(), "value": value, "world": world}))
+    print(json.dumps({"ms": ms, "value": value, "world": world}))
 dist.destroy_process_group()
 """ % ROOT
 
