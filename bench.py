@@ -292,7 +292,11 @@ def stage_work(wl, plan, ratio_k, model=None):
         elif k > 0:
             # k kept values of every unique boundary row, one copy per destination, plus the 16-bit positions
             work["compress"] += nb * k * es + H * k * es + index + nb * k * 2
-            work["decompress"] += H * (k * es + F * es)
+            if 8 * k <= F and F <= 384:
+                # the receiver keeps (value, position) pairs, not dense rows (4 bytes per bf16 pair, 8 per fp32 pair)
+                work["decompress"] += H * (k * es + k * (4 if wl.bf16 else 8)) + nb * k * 2
+            else:
+                work["decompress"] += H * (k * es + F * es)
             work["compress_bwd"] += nb * k * 2       # 16-bit kept positions, once per boundary row
         Hl = H if k > 0 else 0                        # no communication: the halo slots do not exist
         work["spmm"] += nnz_f * 4 + (n + Hl) * F * es + n * F * es + (n + 1) * 8
