@@ -509,7 +509,7 @@ def gemm_layers(model, wl, ks, steps, pk, spans):
             note = None
             if st == "gemm_dx" and narrow_backward(wl, model, l):
                 k = ks[l]
-                slot_gemm = not (k < F and k <= 8 and Fo <= 64)
+                slot_gemm = not (k < F and k <= 16 and Fo <= 64)
                 if slot_gemm and k > 0:
                     flop += 2.0 * H * F * Fo
                 note = "narrow backward: rows n (concatenated K)%s" % (" + the H halo-slot rows" if slot_gemm else "")

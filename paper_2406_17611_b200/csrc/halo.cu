@@ -355,18 +355,20 @@ __global__ void __launch_bounds__(256) select_slots_kernel(const E *__restrict__
 }
 
 // ------------------------------------------------------------------------------------------
-// Backward, receiver side, narrow layers in compressed epochs with at most 8 kept entries (bf16).  The
+// Backward, receiver side, narrow layers in compressed epochs with at most 16 kept entries (bf16).  The
 // gradient row of a halo slot is (slot sum of dZ) W_neigh^T, F_in wide, but only its k kept entries are
 // returned to the owner: entry m is the dot product of the slot's F_out-wide sum with row pi(m) of W_neigh.
-// One thread per slot: the sum is read once into registers, the k positions come as one 16-byte read of the
-// call's table, W_neigh sits in shared memory as F_in rows of bf16 pairs (row stride odd in words, so that
-// the lanes of a warp, which read different rows, spread over the banks), and the 8 packed values of the
-// slot leave as one 16-byte store.  fp32 accumulation, results rounded to bf16 as a GEMM epilogue would.
-// NVO: 16-byte chunks of a row of sums.
+// One thread per slot: the sum is read once into registers, the positions come eight at a time as 16-byte
+// reads of the call's table, W_neigh sits in shared memory as F_in rows of bf16 pairs (row stride odd in
+// words, so that the lanes of a warp, which read different rows, spread over the banks), and every 8 packed
+// values of the slot leave as one 16-byte store.  fp32 accumulation, results rounded to bf16 as a GEMM
+// epilogue would.  Against the dense product (H x F_in values written, read again and picked from: 10 GB
+// each way on the 2.45M-node workload) this is k F_out multiply-adds and k F_out / 2 shared-memory words per
+// slot.  NVO: 16-byte chunks of a row of sums; kv: 16-byte chunks of a packed row.
 template <int NVO>
 __global__ void __launch_bounds__(256) slot_kept_product_kernel(const uint4 *__restrict__ Gh4, int64_t ldg4, int F_out,
                                                                 const __nv_bfloat16 *__restrict__ W, int F_in, int k,
-                                                                int H, uint4 *__restrict__ packed4,
+                                                                int H, uint4 *__restrict__ packed4, int kv,
                                                                 const uint16_t *__restrict__ wpos, int64_t wstride,
                                                                 const int32_t *__restrict__ slot_src) {
   extern __shared__ uint32_t w_pairs[];
@@ -381,8 +383,7 @@ __global__ void __launch_bounds__(256) slot_kept_product_kernel(const uint4 *__r
   }
   __syncthreads();
   for (int slot = blockIdx.x * blockDim.x + threadIdx.x; slot < H; slot += gridDim.x * blockDim.x) {
-    const uint4 pw = __ldg(reinterpret_cast<const uint4 *>(wpos + (int64_t)__ldg(slot_src + slot) * wstride));
-    const uint32_t ps[4] = {pw.x, pw.y, pw.z, pw.w};
+    const uint4 *prow = reinterpret_cast<const uint4 *>(wpos + (int64_t)__ldg(slot_src + slot) * wstride);
     float g[NVO * 8];
 #pragma unroll
     for (int i = 0; i < NVO; ++i) {
@@ -391,21 +392,25 @@ __global__ void __launch_bounds__(256) slot_kept_product_kernel(const uint4 *__r
 #pragma unroll
       for (int j = 0; j < 8; ++j) g[i * 8 + j] = i * 8 + j < F_out ? f[j] : 0.f;
     }
-    float acc[8];
+    for (int c = 0; c * 8 < k; ++c) {
+      const uint4 pw = __ldg(prow + c);
+      const uint32_t ps[4] = {pw.x, pw.y, pw.z, pw.w};
+      float acc[8];
 #pragma unroll
-    for (int m = 0; m < 8; ++m) {
-      acc[m] = 0.f;
-      if (m < k) {
-        const uint32_t *wr = w_pairs + ((ps[m >> 1] >> ((m & 1) * 16)) & 0xFFFFu) * kRowWords;
+      for (int m = 0; m < 8; ++m) {
+        acc[m] = 0.f;
+        if (c * 8 + m < k) {   // table entries at or beyond k are not defined
+          const uint32_t *wr = w_pairs + ((ps[m >> 1] >> ((m & 1) * 16)) & 0xFFFFu) * kRowWords;
 #pragma unroll
-        for (int j = 0; j < NW; ++j) {
-          const uint32_t wj = wr[j];
-          acc[m] = fmaf(g[2 * j], __uint_as_float(wj << 16), acc[m]);
-          acc[m] = fmaf(g[2 * j + 1], __uint_as_float(wj & 0xFFFF0000u), acc[m]);
+          for (int j = 0; j < NW; ++j) {
+            const uint32_t wj = wr[j];
+            acc[m] = fmaf(g[2 * j], __uint_as_float(wj << 16), acc[m]);
+            acc[m] = fmaf(g[2 * j + 1], __uint_as_float(wj & 0xFFFF0000u), acc[m]);
+          }
         }
       }
+      packed4[(int64_t)slot * kv + c] = pack16(acc, __nv_bfloat16());
     }
-    packed4[slot] = pack16(acc, __nv_bfloat16());
   }
 }
 
@@ -711,10 +716,12 @@ int varco_launch_select_slots(const varco_plan *pl, const void *Gh, int64_t ldg,
   return VARCO_OK;
 }
 
-// Kept entries of the slot gradient rows straight from the slot sums of a narrow layer (bf16, k <= 8):
-// packed[slot][m] = Gh[slot] . W_neigh[pi(m)], m < k; packed rows of 8 values.
+// Kept entries of the slot gradient rows straight from the slot sums of a narrow layer (bf16, k <= 16; the
+// lanes of a warp read different rows of W_neigh, so the shared-memory reads collide and at k = 32 the dense
+// product followed by a pick is the faster way again):
+// packed[slot][m] = Gh[slot] . W_neigh[pi(m)], m < k; packed rows of kstride (a multiple of 8) values.
 bool varco_slot_kept_product_supported(int F_in, int F_out, int k, varco_dtype_t dt) {
-  if (dt != VARCO_BF16 || F_out > 64 || k > 8) return false;
+  if (dt != VARCO_BF16 || F_out > 64 || k > 16) return false;
   const int nvo = ((F_out + 7) / 8 + 1) / 2 * 2;
   return (size_t)F_in * (nvo * 4 + 1) * 4 <= 48 * 1024;
 }
@@ -724,7 +731,7 @@ int varco_launch_slot_kept_product(const varco_plan *pl, const void *Gh, int64_t
                                    int64_t wstride, cudaStream_t st) {
   if (pl->H == 0) return VARCO_OK;
   if (!wpos || !varco_slot_kept_product_supported(F_in, F_out, k, VARCO_BF16) || ldg % 8 != 0 || ldg < F_out ||
-      kstride != 8 || wstride % 8 != 0)
+      kstride % 8 != 0 || kstride < k || wstride % 8 != 0)
     return VARCO_INVALID_ARG;
   const int nvo = ((F_out + 7) / 8 + 1) / 2 * 2;   // 2, 4, 6 or 8 chunks
   int dev = 0, sms = 148;
@@ -735,7 +742,8 @@ int varco_launch_slot_kept_product(const varco_plan *pl, const void *Gh, int64_t
   const unsigned grid = (unsigned)(want < (int64_t)sms * 8 ? want : (int64_t)sms * 8);
 #define VARCO_SKP(N)                                                                                               \
   slot_kept_product_kernel<N><<<grid, 256, smem, st>>>((const uint4 *)Gh, ldg / 8, F_out, (const __nv_bfloat16 *)W_neigh, \
-                                                       F_in, k, (int)pl->H, (uint4 *)packed, wpos, wstride,           \
+                                                       F_in, k, (int)pl->H, (uint4 *)packed, (int)(kstride / 8),     \
+                                                       wpos, wstride,                                                \
                                                        pl->d.slot_src)
   if (nvo == 2) VARCO_SKP(2);
   else if (nvo == 4) VARCO_SKP(4);

@@ -913,7 +913,8 @@ template <> struct SparsePair<__nv_bfloat16> {
 };
 
 // halo entries [0, len) of one row: sacc[pos] += w * value for the k pairs of every entry's slot
-template <typename T, int G>
+// (SUM: every weight is 1 and the weights are not read; the caller scales the finished row)
+template <typename T, int G, bool SUM = false>
 __device__ __forceinline__ void accumulate_sparse(const int32_t *__restrict__ colp, const float *__restrict__ valp,
                                                   int len, const typename SparsePair<T>::type *__restrict__ pairs,
                                                   int64_t pstride, int k, int split, float *sacc, int gl,
@@ -923,29 +924,36 @@ __device__ __forceinline__ void accumulate_sparse(const int32_t *__restrict__ co
     const int cnt = min(G, len - base);
     const int mine = base + min(gl, cnt - 1);
     const int myc = __ldg(colp + mine);
-    const float myw = gl < cnt ? __ldg(valp + mine) : 0.f;
+    const float myw = SUM ? 1.f : (gl < cnt ? __ldg(valp + mine) : 0.f);
     if (k <= G) {
-      // one pair per lane and entry: fetch four entries ahead of the shared-memory updates
-      for (int t = 0; t < cnt; t += 4) {
-        P p[4];
-        float w[4];
+      // one pair per lane and entry: fetch kAhead entries ahead of the shared-memory updates
+      constexpr int kAhead = G >= 8 ? 8 : 4;
+      for (int t = 0; t < cnt; t += kAhead) {
+        P p[kAhead];
+        float w[kAhead];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kAhead; ++u) {
           const int slot = __shfl_sync(gmask, myc, t + u, G) - split;
-          w[u] = __shfl_sync(gmask, myw, t + u, G);
+          // past the end of a ragged batch the lane re-reads the last entry with weight 0
+          w[u] = SUM ? (t + u < cnt ? 1.f : 0.f) : __shfl_sync(gmask, myw, t + u, G);
           p[u] = VARCO_DBG_OK(slot, nslots, 11) ? __ldg(pairs + (int64_t)slot * pstride + min(gl, k - 1)) : P();
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (gl < k && VARCO_DBG_OK(SparsePair<T>::pos(p[u]), width, 13))
-            sacc[SparsePair<T>::pos(p[u])] += w[u] * SparsePair<T>::val(p[u]);
+        for (int u = 0; u < kAhead; ++u) {
+          if (gl < k && VARCO_DBG_OK(SparsePair<T>::pos(p[u]), width, 13)) {
+            if (SUM) {
+              if (w[u] != 0.f) sacc[SparsePair<T>::pos(p[u])] += SparsePair<T>::val(p[u]);
+            } else {
+              sacc[SparsePair<T>::pos(p[u])] += w[u] * SparsePair<T>::val(p[u]);
+            }
+          }
           __syncwarp(gmask);
         }
       }
     } else {
       for (int t = 0; t < cnt; ++t) {
         const int slot = __shfl_sync(gmask, myc, t, G) - split;
-        const float w = __shfl_sync(gmask, myw, t, G);
+        const float w = SUM ? 1.f : __shfl_sync(gmask, myw, t, G);
         const P *pr = pairs + (int64_t)slot * pstride;
         if (VARCO_DBG_OK(slot, nslots, 11))
           for (int m = gl; m < k; m += G) {
@@ -959,18 +967,25 @@ __device__ __forceinline__ void accumulate_sparse(const int32_t *__restrict__ co
 }
 
 // One group per row (normal and short classes).  Shared memory: F floats per group.
-template <typename T, int G, int NCH, bool FULL>
-__global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
+// SUM (mean aggregation): the local rows are added unweighted, the pairs likewise, and the finished row is
+// scaled by 1 / deg once.
+// The group is as narrow as the kept count allows (8 lanes for k <= 8, 16 for k <= 16): a pair update occupies k
+// lanes of a group, so a 32-lane group at k = 4 would leave seven lanes in eight idle through the remote part,
+// which is most of the entries on a 16-way partition.
+// (eight pairs in flight per lane: the one-chunk kernels need a few registers more than five resident blocks leave)
+constexpr int sparse_blocks_per_sm(int nch) { return nch == 1 ? 4 : 1; }
+
+template <typename T, int G, int NCH, int UNR, bool FULL, bool SUM>
+__global__ void __launch_bounds__(256, sparse_blocks_per_sm(NCH))
     spmm_sparse_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ nloc,
                        const int32_t *__restrict__ col, const float *__restrict__ val, RowClass rc, GatherSrc gs,
                        const typename SparsePair<T>::type *__restrict__ pairs, int64_t pstride, int k,
-                       T *__restrict__ O, int64_t ldo, int nv) {
+                       const float *__restrict__ row_scale, T *__restrict__ O, int64_t ldo, int nv) {
   extern __shared__ float sparse_acc[];
   constexpr int V = ElemTraits<T>::kVec;
   const int task = (blockIdx.x * blockDim.x + threadIdx.x) / G;
   const int grp = threadIdx.x / G, gl = threadIdx.x % G;
-  const unsigned lane = threadIdx.x % 32;
-  const unsigned gmask = (G == 32) ? 0xFFFFFFFFu : (((1u << G) - 1u) << (lane & ~(unsigned)(G - 1)));
+  const unsigned gmask = group_mask<G>();
   float *sacc = sparse_acc + (size_t)grp * nv * V;
   if (task >= rc.count) return;
   for (int c = gl; c < nv * V; c += G) sacc[c] = 0.f;
@@ -984,16 +999,26 @@ __global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
 #pragma unroll
     for (int j = 0; j < V; ++j) acc[i][j] = 0.f;
   __syncwarp(gmask);
-  if (nl > 0) accumulate_range<T, G, NCH, 4, FULL>(col + e0, val + e0, nl, gs, 0, nv, gl, gmask, acc);
-  if (len > nl) accumulate_sparse<T, G>(col + e0 + nl, val + e0 + nl, len - nl, pairs, pstride, k, gs.split, sacc, gl, gmask,
-                                       gs.nsrc - gs.split, nv * V);
+  if (nl > 0) {
+    if (SUM)
+      sum_range<T, G, NCH, UNR, FULL>(col + e0, nl, gs.b0 + gl, gs.ld0, nv, gl, gmask, acc, 0, gs.split);
+    else
+      accumulate_range<T, G, NCH, UNR, FULL>(col + e0, val + e0, nl, gs, 0, nv, gl, gmask, acc);
+  }
+  if (len > nl)
+    accumulate_sparse<T, G, SUM>(col + e0 + nl, val + e0 + nl, len - nl, pairs, pstride, k, gs.split, sacc, gl, gmask,
+                                 gs.nsrc - gs.split, nv * V);
+  const float scale = SUM ? __ldg(row_scale + r) : 1.f;
   uint4 *dst = reinterpret_cast<uint4 *>(O + (int64_t)r * ldo);
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
     const int ch = gl + i * G;
     if (FULL || ch < nv) {
 #pragma unroll
-      for (int j = 0; j < V; ++j) acc[i][j] += sacc[ch * V + j];
+      for (int j = 0; j < V; ++j) {
+        acc[i][j] += sacc[ch * V + j];
+        if (SUM) acc[i][j] *= scale;
+      }
       dst[ch] = pack16(acc[i], T());
     }
   }
@@ -1001,8 +1026,8 @@ __global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
 
 // Hubs: one CTA per row; every warp takes a contiguous share of the local and of the halo entries and
 // owns one shared-memory row; the rows are added in warp order.
-template <typename T, int NCH, bool FULL>
-__global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
+template <typename T, int NCH, int GK, bool FULL>
+__global__ void __launch_bounds__(256, sparse_blocks_per_sm(NCH))
     spmm_sparse_hub_kernel(const int64_t *__restrict__ rp, const int32_t *__restrict__ nloc,
                            const int32_t *__restrict__ col, const float *__restrict__ val, RowClass rc, GatherSrc gs,
                            const typename SparsePair<T>::type *__restrict__ pairs, int64_t pstride, int k,
@@ -1012,8 +1037,12 @@ __global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int nwarps = blockDim.x / 32;
   const int rowf = nv * V;
-  float *sacc = sparse_acc + (size_t)warp * rowf;
-  for (int c = lane; c < rowf; c += 32) sacc[c] = 0.f;
+  // the halo entries are walked by groups of GK lanes (GK >= k where k <= 32), every group with a row of its own
+  constexpr int kSub = 32 / GK;
+  const int gi = lane / GK, gl = lane % GK;
+  float *wacc = sparse_acc + (size_t)warp * kSub * rowf;   // the warp's kSub rows; the first also takes the local sums
+  float *sacc = wacc + (size_t)gi * rowf;
+  for (int c = lane; c < kSub * rowf; c += 32) wacc[c] = 0.f;
   const int r = __ldg(rc.rows + blockIdx.x);
   const int64_t e0 = rp[r];
   const int len = (int)(rp[r + 1] - e0);
@@ -1032,16 +1061,22 @@ __global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
   int b0, b1;
   share(nl, b0, b1);
   if (b1 > b0) accumulate_range<T, 32, NCH, 4, FULL>(col + e0 + b0, val + e0 + b0, b1 - b0, gs, 0, nv, lane, 0xFFFFFFFFu, acc);
-  share(len - nl, b0, b1);
+  {
+    const int total = len - nl, shares = nwarps * kSub, mine = warp * kSub + gi;
+    const int per = ((total + shares - 1) / shares + GK - 1) / GK * GK;
+    b0 = min(total, mine * per);
+    b1 = min(total, b0 + per);
+  }
   if (b1 > b0)
-    accumulate_sparse<T, 32>(col + e0 + nl + b0, val + e0 + nl + b0, b1 - b0, pairs, pstride, k, gs.split, sacc, lane,
-                             0xFFFFFFFFu, gs.nsrc - gs.split, nv * V);
+    accumulate_sparse<T, GK>(col + e0 + nl + b0, val + e0 + nl + b0, b1 - b0, pairs, pstride, k, gs.split, sacc, gl,
+                             group_mask<GK>(), gs.nsrc - gs.split, nv * V);
+  __syncwarp();
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
     const int ch = lane + i * 32;
     if (FULL || ch < nv)
 #pragma unroll
-      for (int j = 0; j < V; ++j) sacc[ch * V + j] += acc[i][j];
+      for (int j = 0; j < V; ++j) wacc[ch * V + j] += acc[i][j];
   }
   __syncthreads();
   uint4 *dst = reinterpret_cast<uint4 *>(O + (int64_t)r * ldo);
@@ -1049,68 +1084,89 @@ __global__ void __launch_bounds__(256, rows_blocks_per_sm(NCH))
     float f[V];
 #pragma unroll
     for (int j = 0; j < V; ++j) f[j] = 0.f;
-    for (int w = 0; w < nwarps; ++w)
+    for (int w = 0; w < nwarps * kSub; ++w)
 #pragma unroll
       for (int j = 0; j < V; ++j) f[j] += sparse_acc[(size_t)w * rowf + ch * V + j];
     dst[ch] = pack16(f, T());
   }
 }
 
-template <typename T, int G, int NCH>
+template <typename T, int G, int NCH, int UNR>
 int launch_sparse_rows(const SpmmArgs &a, const RowClass &rc, const int32_t *nloc, const void *pairs, int64_t pstride,
-                       int k, cudaStream_t st) {
+                       int k, const float *row_scale, cudaStream_t st) {
   if (rc.count == 0) return VARCO_OK;
   constexpr int V = ElemTraits<T>::kVec;
   typedef typename SparsePair<T>::type P;
   const int threads = 256;
   const size_t smem = (size_t)(threads / G) * a.nv * V * sizeof(float);
   dim3 grid((unsigned)(((int64_t)rc.count * G + threads - 1) / threads));
-  if (a.nv == G * NCH)
-    spmm_sparse_kernel<T, G, NCH, true><<<grid, threads, smem, st>>>(a.rp, nloc, a.col, a.val, rc, gather_src<T>(a),
-                                                                     (const P *)pairs, pstride, k, (T *)a.O0, a.ldo0,
-                                                                     a.nv);
-  else
-    spmm_sparse_kernel<T, G, NCH, false><<<grid, threads, smem, st>>>(a.rp, nloc, a.col, a.val, rc, gather_src<T>(a),
-                                                                      (const P *)pairs, pstride, k, (T *)a.O0, a.ldo0,
-                                                                      a.nv);
+  const bool full = a.nv == G * NCH;
+#define VARCO_SPARSE_LAUNCH(FULL, SUM)                                                                              \
+  spmm_sparse_kernel<T, G, NCH, UNR, FULL, SUM><<<grid, threads, smem, st>>>(                                       \
+      a.rp, nloc, a.col, a.val, rc, gather_src<T>(a), (const P *)pairs, pstride, k, row_scale, (T *)a.O0, a.ldo0, a.nv)
+  if (row_scale) {
+    if (full)
+      VARCO_SPARSE_LAUNCH(true, true);
+    else
+      VARCO_SPARSE_LAUNCH(false, true);
+  } else {
+    if (full)
+      VARCO_SPARSE_LAUNCH(true, false);
+    else
+      VARCO_SPARSE_LAUNCH(false, false);
+  }
+#undef VARCO_SPARSE_LAUNCH
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
-template <typename T, int NCH>
+template <typename T, int NCH, int GK>
 int launch_sparse_hubs(const SpmmArgs &a, const int32_t *nloc, const void *pairs, int64_t pstride, int k,
                        cudaStream_t st) {
   if (a.hubs.count == 0) return VARCO_OK;
   constexpr int V = ElemTraits<T>::kVec;
   typedef typename SparsePair<T>::type P;
-  const size_t row_bytes = (size_t)a.nv * V * sizeof(float);
+  const size_t row_bytes = (size_t)(32 / GK) * a.nv * V * sizeof(float);   // per warp: one row per group of GK lanes
   int warps = 8;
   while (warps > 1 && warps * row_bytes > 48 * 1024) warps /= 2;
+  if (warps * row_bytes > 48 * 1024) return VARCO_UNSUPPORTED;
   if (a.nv == 32 * NCH)
-    spmm_sparse_hub_kernel<T, NCH, true><<<a.hubs.count, warps * 32, warps * row_bytes, st>>>(
+    spmm_sparse_hub_kernel<T, NCH, GK, true><<<a.hubs.count, warps * 32, warps * row_bytes, st>>>(
         a.rp, nloc, a.col, a.val, a.hubs, gather_src<T>(a), (const P *)pairs, pstride, k, (T *)a.O0, a.ldo0, a.nv);
   else
-    spmm_sparse_hub_kernel<T, NCH, false><<<a.hubs.count, warps * 32, warps * row_bytes, st>>>(
+    spmm_sparse_hub_kernel<T, NCH, GK, false><<<a.hubs.count, warps * 32, warps * row_bytes, st>>>(
         a.rp, nloc, a.col, a.val, a.hubs, gather_src<T>(a), (const P *)pairs, pstride, k, (T *)a.O0, a.ldo0, a.nv);
   VARCO_KERNEL_LAUNCHED();
   return VARCO_OK;
 }
 
-// lanes per row for the ordinary class / the short class, by row width in chunks (nv <= 64 only)
+// Lanes per row for the ordinary class / the short class, by row width in chunks (nv <= 64 only) and by the
+// kept count; UNR x NCH 16-byte gathers of the local part in flight per lane.  row_scale != nullptr: mean
+// aggregation as unweighted sums (hub rows keep the weighted kernel: the same sums, scaled entry by entry).
 template <typename T>
 int dispatch_sparse(const SpmmArgs &a, const int32_t *nloc, const void *pairs, int64_t pstride, int k,
-                    cudaStream_t st) {
+                    const float *row_scale, cudaStream_t st) {
   const int w = a.nv;
-#define VARCO_SPARSE(G, NCH, GS, NCHS)                                                               \
-  do {                                                                                               \
-    if (int rc = launch_sparse_hubs<T, (NCH * G + 31) / 32>(a, nloc, pairs, pstride, k, st)) return rc; \
-    if (int rc = launch_sparse_rows<T, G, NCH>(a, a.normal, nloc, pairs, pstride, k, st)) return rc;  \
-    return launch_sparse_rows<T, GS, NCHS>(a, a.shorts, nloc, pairs, pstride, k, st);                 \
+#define VARCO_SPARSE(G, NCH, UNR, GS, NCHS)                                                                     \
+  do {                                                                                                          \
+    if (int rc = launch_sparse_hubs<T, (NCH * G + 31) / 32, G>(a, nloc, pairs, pstride, k, st)) return rc;      \
+    if (int rc = launch_sparse_rows<T, G, NCH, UNR>(a, a.normal, nloc, pairs, pstride, k, row_scale, st)) return rc; \
+    return launch_sparse_rows<T, GS, NCHS, 2>(a, a.shorts, nloc, pairs, pstride, k, row_scale, st);             \
   } while (0)
-  if (w <= 8) VARCO_SPARSE(8, 1, 8, 1);
-  if (w <= 16) VARCO_SPARSE(16, 1, 8, 2);
-  if (w <= 32) VARCO_SPARSE(32, 1, 8, 4);
-  if (w <= 64) VARCO_SPARSE(32, 2, 16, 4);
+  if (w <= 8) VARCO_SPARSE(8, 1, 4, 8, 1);
+  if (w <= 16) {
+    if (k <= 8) VARCO_SPARSE(8, 2, 4, 8, 2);
+    VARCO_SPARSE(16, 1, 4, 8, 2);
+  }
+  if (w <= 32) {
+    if (k <= 8) VARCO_SPARSE(8, 4, 2, 8, 4);
+    if (k <= 16) VARCO_SPARSE(16, 2, 4, 8, 4);
+    VARCO_SPARSE(32, 1, 4, 8, 4);
+  }
+  if (w <= 64) {
+    if (k <= 16) VARCO_SPARSE(16, 4, 2, 16, 4);
+    VARCO_SPARSE(32, 2, 4, 16, 4);
+  }
 #undef VARCO_SPARSE
   return VARCO_UNSUPPORTED;
 }
@@ -1230,8 +1286,9 @@ int varco_launch_spmm_fwd_sparse(const varco_plan *pl, const void *X, int64_t ld
   a.nv = (F + V - 1) / V;
   a.panels = 1;
   a.nv_panel = a.nv;
-  return dt == VARCO_F32 ? dispatch_sparse<float>(a, pl->d.nloc, pairs, pstride, k, st)
-                         : dispatch_sparse<__nv_bfloat16>(a, pl->d.nloc, pairs, pstride, k, st);
+  const float *row_scale = (!pl->row_scale.empty() && ldx % V == 0) ? pl->d.row_scale : nullptr;
+  return dt == VARCO_F32 ? dispatch_sparse<float>(a, pl->d.nloc, pairs, pstride, k, row_scale, st)
+                         : dispatch_sparse<__nv_bfloat16>(a, pl->d.nloc, pairs, pstride, k, row_scale, st);
 }
 
 // Transposed aggregation: for a source u, g_u = sum over the rows i that use it of s_iu dAgg[i];

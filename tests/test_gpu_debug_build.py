@@ -22,7 +22,7 @@ from helpers import LayerCase, close, dev_weights, host64, to_device_rows, to_ho
 assert vb.varco_debug_status() == (True, 0)
 orc = oracle.Oracle()
 for name, scale, layer, ratio in [("c1", 0.2, 0, (4, 1)), ("c1", 0.2, 1, (1, 1)), ("c2r", 0.01, 1, (16, 1)),
-                                  ("c3", 0.002, 1, (1, 1)), ("c3", 0.002, 2, (64, 1)), ("c3", 0.002, 0, (1, 0)),
+                                  ("c3", 0.002, 1, (1, 1)), ("c3", 0.002, 2, (64, 1)), ("c3", 0.002, 2, (4, 1)), ("c3", 0.002, 0, (1, 0)),
                                   ("c4", 0.01, 0, (8, 1))]:
     case = LayerCase(orc, synth.make_workload(name, scale))
     wl, dt = case.wl, case.dtype
