@@ -298,6 +298,11 @@ def stage_work(wl, plan, ratio_k, model=None):
             else:
                 work["decompress"] += H * (k * es + F * es)
             work["compress_bwd"] += nb * k * 2       # 16-bit kept positions, once per boundary row
+            if model is not None and narrow_backward(wl, model, l):
+                # narrow layer: the slot gradients are compressed in a pass of their own -- from the F_out-wide
+                # slot sums (k <= 16: one dot product per kept entry) or from the dense F-wide product
+                src = Fo if (k <= 16 and Fo <= 64) else F
+                work["compress_bwd"] += H * (src * es + k * es + 4 + k * 2)
         Hl = H if k > 0 else 0                        # no communication: the halo slots do not exist
         work["spmm"] += nnz_f * 4 + (n + Hl) * F * es + n * F * es + (n + 1) * 8
         Fb = Fo if model is not None and narrow_backward(wl, model, l) else F

@@ -359,10 +359,10 @@ __global__ void __launch_bounds__(256) select_slots_kernel(const E *__restrict__
 // gradient row of a halo slot is (slot sum of dZ) W_neigh^T, F_in wide, but only its k kept entries are
 // returned to the owner: entry m is the dot product of the slot's F_out-wide sum with row pi(m) of W_neigh.
 // One thread per slot: the sum is read once into registers, the positions come eight at a time as 16-byte
-// reads of the call's table, W_neigh sits in shared memory as F_in rows of bf16 pairs (row stride odd in
-// words, so that the lanes of a warp, which read different rows, spread over the banks), and every 8 packed
-// values of the slot leave as one 16-byte store.  fp32 accumulation, results rounded to bf16 as a GEMM
-// epilogue would.  Against the dense product (H x F_in values written, read again and picked from: 10 GB
+// reads of the call's table, W_neigh sits in shared memory as F_in rows of bf16 pairs (16-byte aligned rows an
+// odd number of 16-byte units apart, read with 16-byte loads: the lanes of a warp read different rows), and
+// every 8 packed values of the slot leave as one 16-byte store.  fp32 accumulation, results rounded to bf16 as a
+// GEMM epilogue would.  Against the dense product (H x F_in values written, read again and picked from: 10 GB
 // each way on the 2.45M-node workload) this is k F_out multiply-adds and k F_out / 2 shared-memory words per
 // slot.  NVO: 16-byte chunks of a row of sums; kv: 16-byte chunks of a packed row.
 template <int NVO>
@@ -371,9 +371,9 @@ __global__ void __launch_bounds__(256) slot_kept_product_kernel(const uint4 *__r
                                                                 int H, uint4 *__restrict__ packed4, int kv,
                                                                 const uint16_t *__restrict__ wpos, int64_t wstride,
                                                                 const int32_t *__restrict__ slot_src) {
-  extern __shared__ uint32_t w_pairs[];
+  extern __shared__ __align__(16) uint32_t w_pairs[];
   constexpr int NW = NVO * 4;          // words (pairs) per row
-  constexpr int kRowWords = NW + 1;
+  constexpr int kRowWords = NW + 4;    // rows 16-byte aligned, an odd number of 16-byte units apart
   const uint16_t *Wbits = reinterpret_cast<const uint16_t *>(W);
   for (int i = threadIdx.x; i < F_in * NW; i += blockDim.x) {
     const int f = i / NW, j = i % NW;
@@ -400,12 +400,17 @@ __global__ void __launch_bounds__(256) slot_kept_product_kernel(const uint4 *__r
       for (int m = 0; m < 8; ++m) {
         acc[m] = 0.f;
         if (c * 8 + m < k) {   // table entries at or beyond k are not defined
-          const uint32_t *wr = w_pairs + ((ps[m >> 1] >> ((m & 1) * 16)) & 0xFFFFu) * kRowWords;
+          const uint4 *wr = reinterpret_cast<const uint4 *>(w_pairs + ((ps[m >> 1] >> ((m & 1) * 16)) & 0xFFFFu) * kRowWords);
 #pragma unroll
-          for (int j = 0; j < NW; ++j) {
-            const uint32_t wj = wr[j];
-            acc[m] = fmaf(g[2 * j], __uint_as_float(wj << 16), acc[m]);
-            acc[m] = fmaf(g[2 * j + 1], __uint_as_float(wj & 0xFFFF0000u), acc[m]);
+          for (int jq = 0; jq < NVO; ++jq) {
+            const uint4 wq = wr[jq];
+            const uint32_t wj[4] = {wq.x, wq.y, wq.z, wq.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int j = jq * 4 + i;
+              acc[m] = fmaf(g[2 * j], __uint_as_float(wj[i] << 16), acc[m]);
+              acc[m] = fmaf(g[2 * j + 1], __uint_as_float(wj[i] & 0xFFFF0000u), acc[m]);
+            }
           }
         }
       }
@@ -723,7 +728,7 @@ int varco_launch_select_slots(const varco_plan *pl, const void *Gh, int64_t ldg,
 bool varco_slot_kept_product_supported(int F_in, int F_out, int k, varco_dtype_t dt) {
   if (dt != VARCO_BF16 || F_out > 64 || k > 16) return false;
   const int nvo = ((F_out + 7) / 8 + 1) / 2 * 2;
-  return (size_t)F_in * (nvo * 4 + 1) * 4 <= 48 * 1024;
+  return (size_t)F_in * (nvo * 4 + 4) * 4 <= 48 * 1024;
 }
 
 int varco_launch_slot_kept_product(const varco_plan *pl, const void *Gh, int64_t ldg, int F_out, const void *W_neigh,
@@ -737,7 +742,7 @@ int varco_launch_slot_kept_product(const varco_plan *pl, const void *Gh, int64_t
   int dev = 0, sms = 148;
   VARCO_CUDA_CHECK(cudaGetDevice(&dev));
   VARCO_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  const size_t smem = (size_t)F_in * (nvo * 4 + 1) * 4;
+  const size_t smem = (size_t)F_in * (nvo * 4 + 4) * 4;
   const int64_t want = (pl->H + 255) / 256;
   const unsigned grid = (unsigned)(want < (int64_t)sms * 8 ? want : (int64_t)sms * 8);
 #define VARCO_SKP(N)                                                                                               \

@@ -132,6 +132,9 @@ int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   // receiver, so "send buffer -> receive buffer" is folded into the write address.  At full
   // communication the row travels whole and in order: one gather-copy fills the halo slots.
   const int64_t kstride = round_up64(k, V);
+  // rows of the position table are as long as this call's kept count needs (a multiple of 8 entries), not F_in:
+  // at high ratios the table of all boundary rows then fits L2 and a 16-byte read of it costs one sector, not a line
+  const int64_t wstride = round_up64(k > 0 ? k : 1, 8);
   // Compressed epochs with at most a quarter of a row kept: the receiver keeps (value, position)
   // pairs instead of rows that are mostly zeros, and the aggregation reads k pairs per remote
   // neighbour instead of F elements.
@@ -144,14 +147,14 @@ int varco_layer_fwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   } else {
     {
       StageTimer t(plan, VARCO_STAGE_COMPRESS, stream);
-      rc = varco_launch_compress_rows(plan, X, desc->ld_in, F_in, k, dt, key, packed, kstride, 0, wpos, L.wstride, st);
+      rc = varco_launch_compress_rows(plan, X, desc->ld_in, F_in, k, dt, key, packed, kstride, 0, wpos, wstride, st);
     }
     if (rc != VARCO_OK) return rc;
     StageTimer t(plan, VARCO_STAGE_DECOMPRESS, stream);
     if (sparse)
-      rc = varco_launch_expand_slots(plan, packed, kstride, k, dt, Xhalo, round_up64(k, 4), wpos, L.wstride, st);
+      rc = varco_launch_expand_slots(plan, packed, kstride, k, dt, Xhalo, round_up64(k, 4), wpos, wstride, st);
     else
-      rc = varco_launch_decompress_slots(plan, packed, kstride, 0, F_in, k, dt, key, Xhalo, L.ld_in, wpos, L.wstride,
+      rc = varco_launch_decompress_slots(plan, packed, kstride, 0, F_in, k, dt, key, Xhalo, L.ld_in, wpos, wstride,
                                          st);
   }
   if (rc != VARCO_OK) return rc;
@@ -273,11 +276,14 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   const bool narrow = tc && 2 * L.ld_out <= F_in;
   uint16_t *wpos = reinterpret_cast<uint16_t *>(ws + L.wpos);
   const int64_t kstride = round_up64(k, V);
+  // rows of the position table are as long as this call's kept count needs (a multiple of 8 entries), not F_in:
+  // at high ratios the table of all boundary rows then fits L2 and a 16-byte read of it costs one sector, not a line
+  const int64_t wstride = round_up64(k > 0 ? k : 1, 8);
   if (k > 0 && k < F_in) {
     // the kept positions of every unique boundary row are evaluated once, then used by the compression of
     // the slot gradients and by the owners' add
     StageTimer t(plan, VARCO_STAGE_COMPRESS_BWD, stream);
-    rc = varco_launch_wire_positions(plan, F_in, k, key, wpos, L.wstride, st);
+    rc = varco_launch_wire_positions(plan, F_in, k, key, wpos, wstride, st);
     if (rc != VARCO_OK) return rc;
   }
   if (narrow) {
@@ -307,12 +313,12 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
       // few kept entries: each one is a dot product with one row of W_neigh; the F_in-wide rows never exist
       {
         StageTimer t(plan, VARCO_STAGE_COMPRESS_BWD, stream);
-        rc = varco_launch_slot_kept_product(plan, Gh, L.ld_out, F_out, W_neigh, F_in, k, Ghalo, kstride, wpos, L.wstride,
+        rc = varco_launch_slot_kept_product(plan, Gh, L.ld_out, F_out, W_neigh, F_in, k, Ghalo, kstride, wpos, wstride,
                                             st);
       }
       if (rc != VARCO_OK) return rc;
       StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
-      return varco_launch_scatter_add_rows(plan, Ghalo, kstride, F_in, k, dt, dX, desc->ld_in, wpos, L.wstride, st);
+      return varco_launch_scatter_add_rows(plan, Ghalo, kstride, F_in, k, dt, dX, desc->ld_in, wpos, wstride, st);
     }
     if (k == F_in) {
       StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
@@ -320,11 +326,11 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
     }
     {
       StageTimer t(plan, VARCO_STAGE_COMPRESS_BWD, stream);
-      rc = varco_launch_select_slots(plan, Ghalo, L.ld_in, F_in, k, dt, packed, kstride, wpos, L.wstride, st);
+      rc = varco_launch_select_slots(plan, Ghalo, L.ld_in, F_in, k, dt, packed, kstride, wpos, wstride, st);
     }
     if (rc != VARCO_OK) return rc;
     StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
-    return varco_launch_scatter_add_rows(plan, packed, kstride, F_in, k, dt, dX, desc->ld_in, wpos, L.wstride, st);
+    return varco_launch_scatter_add_rows(plan, packed, kstride, F_in, k, dt, dX, desc->ld_in, wpos, wstride, st);
   }
   {
     StageTimer t(plan, VARCO_STAGE_GEMM_DX, stream);
@@ -341,7 +347,7 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
     StageTimer t(plan, VARCO_STAGE_SPMM_T, stream);
     // k < F: the slot gradients are compressed in the epilogue (no dense slot rows)
     rc = varco_launch_spmm_bwd(plan, dAgg, L.ld_in, F_in, dt, dX, desc->ld_in, sage ? 1 : 0, k > 0 ? Ghalo : nullptr,
-                               L.ld_in, (k > 0 && k < F_in) ? packed : nullptr, kstride, k, key, wpos, L.wstride, st);
+                               L.ld_in, (k > 0 && k < F_in) ? packed : nullptr, kstride, k, key, wpos, wstride, st);
   }
   if (rc != VARCO_OK || k == 0) return rc;   // no communication: no gradient crosses a partition boundary
   // Return of the halo-slot gradients to the owners.  At full communication the slot rows are
@@ -352,7 +358,7 @@ int varco_layer_bwd(const varco_plan_t *plan, const varco_layer_desc_t *desc, co
   }
   {
     StageTimer t(plan, VARCO_STAGE_SCATTER_ADD, stream);
-    rc = varco_launch_scatter_add_rows(plan, packed, kstride, F_in, k, dt, dX, desc->ld_in, wpos, L.wstride, st);
+    rc = varco_launch_scatter_add_rows(plan, packed, kstride, F_in, k, dt, dX, desc->ld_in, wpos, wstride, st);
   }
   return rc;
 }

@@ -973,7 +973,7 @@ __device__ __forceinline__ void accumulate_sparse(const int32_t *__restrict__ co
 // lanes of a group, so a 32-lane group at k = 4 would leave seven lanes in eight idle through the remote part,
 // which is most of the entries on a 16-way partition.
 // (eight pairs in flight per lane: the one-chunk kernels need a few registers more than five resident blocks leave)
-constexpr int sparse_blocks_per_sm(int nch) { return nch == 1 ? 4 : 1; }
+constexpr int sparse_blocks_per_sm(int nch) { return nch == 1 ? 4 : (nch <= 4 ? 3 : 1); }
 
 template <typename T, int G, int NCH, int UNR, bool FULL, bool SUM>
 __global__ void __launch_bounds__(256, sparse_blocks_per_sm(NCH))
